@@ -1,0 +1,156 @@
+/*
+ * rpx — prefix/suffix scoring kernels for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The operations follow the paper's statement of the problem (Section 2.3 "Observation and
+ * Opportunity"; Section 3.1 Phases 1-2; Table 4, rows "Boundary prefix KV" and "Prefix
+ * logprobs"): every model invocation of an RL iteration is split at the first response position
+ * into a response-independent PREFIX (the prompt: visual + text tokens) and a response SUFFIX.
+ * The prefix pass produces boundary KV state and prefix log-probabilities before the responses
+ * exist; the suffix pass consumes the responses together with the retained boundary KV; prefix
+ * and suffix log-probabilities together are the full-sequence values.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers unless marked "host".  Descriptor structs
+ *     (rpx_attn_desc_t, rpx_kv_cache_t) are read on the HOST during the call.
+ *   - The caller owns every buffer (inputs, outputs, cache pool, block table, workspace, status
+ *     word) and must keep it alive until `cuda_stream` has executed the enqueued work.  The
+ *     library allocates no device memory, keeps no state between calls and never synchronises:
+ *     a call only enqueues kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream) of the current device.
+ *   - Packed layouts: a [tokens][heads][head_dim] tensor has head_dim contiguous, heads
+ *     contiguous (stride head_dim) and a caller-given token stride in ELEMENTS.  Sequence s owns
+ *     tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (int32, device, batch+1 entries, cu_seqlens[0]=0).
+ *   - Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *   - Element types: RPX_BF16 tensors are bfloat16; RPX_F32 tensors are float32 and are rounded
+ *     to bf16 (nearest-even) in a pre-pass into the workspace, after which the same bf16
+ *     tensor-core kernels run; outputs then come back as float32.  The KV cache is always bf16.
+ *   - Host-checkable problems (NULL pointer, head counts, head_dim, block size, alignment,
+ *     strides, workspace size, device architecture) return a negative status BEFORE any launch.
+ *     Problems only visible on the device (a kernel-side wait that ran out, an out-of-range
+ *     target id or block id) are written to *device_status (nullable, device int32, zeroed by the
+ *     caller): the first error code wins; the caller reads it after its own synchronisation.
+ *     Every kernel-side wait is bounded: on expiry the kernel records RPX_ERR_TIMEOUT, drains and
+ *     returns; outputs of that call are then undefined.
+ *   - Alignment: every tensor pointer 16-byte aligned; token/row strides multiples of 8 elements.
+ *   - Zero-length sequences, batch == 0 and n_tokens == 0 are legal no-ops.
+ */
+#ifndef RPX_H_
+#define RPX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t rpx_status_t;
+enum {
+    RPX_OK = 0,
+    RPX_ERR_NULL = -1,        /* a required pointer is NULL                                  */
+    RPX_ERR_SHAPE = -2,       /* unsupported or inconsistent sizes                           */
+    RPX_ERR_DTYPE = -3,       /* unknown element type                                        */
+    RPX_ERR_ALIGN = -4,       /* pointer or stride alignment                                 */
+    RPX_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than *_workspace_bytes            */
+    RPX_ERR_ARCH = -6,        /* current device is not compute capability 10.x               */
+    RPX_ERR_CUDA = -7,        /* a CUDA runtime/driver call failed                           */
+    RPX_ERR_DEVICE_DATA = -8, /* (device_status) out-of-range id found in device data        */
+    RPX_ERR_TIMEOUT = -9      /* (device_status) a bounded kernel-side wait expired          */
+};
+
+typedef enum { RPX_BF16 = 0, RPX_F32 = 1 } rpx_dtype_t;
+
+/* Attention problem shape.  head_dim is 64 or 128; num_q_heads % num_kv_heads == 0.
+ * softmax_scale <= 0 selects 1/sqrt(head_dim).  No bias, soft-cap, window or dropout. */
+typedef struct {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;
+    float softmax_scale;
+    rpx_dtype_t dtype; /* element type of q, k, v and out */
+} rpx_attn_desc_t;
+
+/* Paged boundary-KV cache (Table 4, "Boundary prefix KV": produced by the prefix pass, kept in
+ * HBM by the caller, consumed by the suffix pass).
+ *   k_cache, v_cache : bf16 [num_blocks][num_kv_heads][block_size][head_dim], 16-byte aligned
+ *   block_table      : device int32 [batch][block_table_stride]; prefix position t of sequence s
+ *                      lives in slot  block_table[s][t / block_size] * block_size + t % block_size
+ *   block_size       : must be 16 */
+typedef struct {
+    void* k_cache;
+    void* v_cache;
+    int64_t num_blocks;
+    int32_t block_size;
+    const int32_t* block_table;
+    int32_t block_table_stride;
+} rpx_kv_cache_t;
+
+/*
+ * Prefix attention + boundary-KV write (Section 3.1, Phase 1: "prefill the prompt ... produces
+ * ... boundary KV state").  For every sequence s, query head h and prompt position i:
+ *     out[i,h,:] = sum_{j<=i} softmax_j(scale * q[i,h,:].k[j,g,:]) * v[j,g,:],   g = h / group
+ * and, when `cache` is non-NULL, K and V of every prompt token are stored (as bf16) at the
+ * token's slot of the paged cache; slots no token maps to are not touched.
+ *   q [total_tokens][num_q_heads][head_dim], k, v [total_tokens][num_kv_heads][head_dim]
+ *   out [total_tokens][num_q_heads][head_dim] contiguous, element type desc->dtype
+ *   lse (nullable) float32 [total_tokens][num_q_heads]: ln sum_j exp(scale * q.k_j)
+ *   max_seqlen: an upper bound on the longest sequence (sizes the grid).
+ */
+rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                             int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
+                             const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens,
+                             int32_t max_seqlen, const rpx_kv_cache_t* cache, void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, int32_t* device_status,
+                             void* cuda_stream);
+
+/*
+ * Suffix attention over the retained boundary (Section 3.1, Phase 2: "suffixes consume the
+ * responses and their preserved boundaries"; Section 2.3: they "continue from the retained prefix
+ * boundary rather than recomputing the prompt").  Response position r of sequence s (global
+ * position prefix_lens[s] + r) attends to all prefix_lens[s] cached keys and to response keys
+ * 0..r; the result equals rows prefix_lens[s].. of one-pass attention over the whole sequence.
+ *   q, k, v: response tokens only, packed by cu_seqlens_suffix; prefix_lens device int32 [batch]
+ *   cache: required, read-only here (response K/V are NOT appended; they have no later reader)
+ *   max_suffix_len / max_prefix_len: upper bounds (grid sizing only).
+ */
+rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                             int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
+                             const int32_t* cu_seqlens_suffix, const int32_t* prefix_lens, int32_t batch,
+                             int64_t total_suffix_tokens, int32_t max_suffix_len, int32_t max_prefix_len,
+                             const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
+/*
+ * Fused LM-head log-probabilities (Section 3.1: Phase 1 yields "prefix log-probabilities",
+ * Phase 2 the suffix ones; Table 4 "Prefix logprobs").  For every row n:
+ *     z_v = hidden[n,:] . w_vocab[v,:]          (never stored)
+ *     logprobs[n] = z_{target_ids[n]} - ln sum_v exp(z_v)
+ *   hidden [n_tokens][hidden_dim] with row stride in elements; w_vocab [vocab][hidden_dim]
+ *   row-major contiguous; target_ids device int32 [n_tokens]; hidden_dim % 8 == 0.
+ *   logprobs float32 [n_tokens]; lse (nullable) float32 [n_tokens].
+ * A target outside [0, vocab) gives NaN for that row and RPX_ERR_DEVICE_DATA in *device_status.
+ * The kernel is position-agnostic: which (hidden row, next token) pairs form the prefix call and
+ * which the suffix call is the caller's choice.
+ */
+rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
+                                int32_t vocab, rpx_dtype_t dtype, float* logprobs, float* lse,
+                                void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                void* cuda_stream);
+
+/* Workspace sizes in bytes for the calls above (pure host arithmetic; 0 is possible). */
+size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens);
+size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens);
+size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                          rpx_dtype_t dtype);
+
+/* Static string for a status code; never NULL. */
+const char* rpx_status_string(rpx_status_t status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int32_t rpx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RPX_H_ */

@@ -1,0 +1,250 @@
+"""ctypes binding of ``librpx.so`` (the C ABI declared in ``include/rpx.h``).
+
+Only argument marshalling happens here: torch tensors supply device pointers and the current
+stream; every step of the scoring path runs inside the CUDA library.  If the library is missing
+the functions raise — there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librpx.so")
+_lib = None
+
+RPX_BF16, RPX_F32 = 0, 1
+BLOCK_SIZE = 16
+
+EXPORTS = (
+    "rpx_prefix_attn",
+    "rpx_suffix_attn",
+    "rpx_token_logprobs",
+    "rpx_prefix_attn_workspace_bytes",
+    "rpx_suffix_attn_workspace_bytes",
+    "rpx_token_logprobs_workspace_bytes",
+    "rpx_status_string",
+    "rpx_version",
+)
+
+
+class RpxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [
+        ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float),
+        ("dtype", ctypes.c_int32),
+    ]
+
+
+class KvCache(ctypes.Structure):
+    _fields_ = [
+        ("k_cache", ctypes.c_void_p),
+        ("v_cache", ctypes.c_void_p),
+        ("num_blocks", ctypes.c_int64),
+        ("block_size", ctypes.c_int32),
+        ("block_table", ctypes.c_void_p),
+        ("block_table_stride", ctypes.c_int32),
+    ]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load librpx.so (built in-tree by ``paper_2608_14498_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise FileNotFoundError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2608_14498_b200.build` "
+            "(there is no CPU or eager fallback)"
+        )
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lib.rpx_prefix_attn.restype = i32
+    lib.rpx_prefix_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, i64, i64, i64, vp, i32, i64, i32,
+                                    ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
+    lib.rpx_suffix_attn.restype = i32
+    lib.rpx_suffix_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, i64, i64, i64, vp, vp, i32, i64, i32,
+                                    i32, ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs.restype = i32
+    lib.rpx_token_logprobs.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.rpx_prefix_attn_workspace_bytes.restype = sz
+    lib.rpx_prefix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
+    lib.rpx_suffix_attn_workspace_bytes.restype = sz
+    lib.rpx_suffix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
+    lib.rpx_token_logprobs_workspace_bytes.restype = sz
+    lib.rpx_token_logprobs_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    lib.rpx_status_string.restype = ctypes.c_char_p
+    lib.rpx_status_string.argtypes = [i32]
+    lib.rpx_version.restype = i32
+    lib.rpx_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().rpx_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(load_library().rpx_version())
+
+
+# ------------------------------------------------------------------ helpers (torch side)
+def _torch():
+    import torch
+
+    return torch
+
+
+def _dtype_code(t) -> int:
+    torch = _torch()
+    if t.dtype == torch.bfloat16:
+        return RPX_BF16
+    if t.dtype == torch.float32:
+        return RPX_F32
+    raise TypeError(f"rpx tensors are bfloat16 or float32, got {t.dtype}")
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream_ptr(stream) -> int:
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _tok_stride(t) -> int:
+    if t.dim() != 3 or t.stride(2) != 1 or t.stride(1) != t.shape[2]:
+        raise ValueError("expected a [tokens, heads, head_dim] tensor with contiguous heads")
+    return t.stride(0) if t.shape[0] > 1 else t.shape[1] * t.shape[2]
+
+
+def _workspace(nbytes: int, device, workspace):
+    torch = _torch()
+    if workspace is not None:
+        if workspace.numel() * workspace.element_size() < nbytes:
+            raise ValueError(f"workspace too small: need {nbytes} bytes")
+        return workspace
+    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device=device)
+
+
+def _desc(q, k, softmax_scale: float) -> AttnDesc:
+    return AttnDesc(q.shape[1], k.shape[1], q.shape[2], float(softmax_scale), _dtype_code(q))
+
+
+def _cache_struct(cache) -> KvCache:
+    k_cache, v_cache, block_table = cache
+    torch = _torch()
+    if k_cache.dtype != torch.bfloat16 or v_cache.dtype != torch.bfloat16 or block_table.dtype != torch.int32:
+        raise TypeError("cache pools are bfloat16 and the block table is int32")
+    if not (k_cache.is_contiguous() and v_cache.is_contiguous()) or block_table.stride(1) != 1:
+        raise ValueError("cache pools must be contiguous [blocks, kv_heads, 16, head_dim]")
+    return KvCache(k_cache.data_ptr(), v_cache.data_ptr(), k_cache.shape[0], k_cache.shape[2],
+                   block_table.data_ptr(), block_table.stride(0))
+
+
+def prefix_attn_workspace_bytes(num_q_heads, num_kv_heads, head_dim, dtype_code, total_tokens) -> int:
+    d = AttnDesc(num_q_heads, num_kv_heads, head_dim, 0.0, dtype_code)
+    return int(load_library().rpx_prefix_attn_workspace_bytes(ctypes.byref(d), int(total_tokens)))
+
+
+def suffix_attn_workspace_bytes(num_q_heads, num_kv_heads, head_dim, dtype_code, total_tokens) -> int:
+    d = AttnDesc(num_q_heads, num_kv_heads, head_dim, 0.0, dtype_code)
+    return int(load_library().rpx_suffix_attn_workspace_bytes(ctypes.byref(d), int(total_tokens)))
+
+
+def token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype_code) -> int:
+    return int(load_library().rpx_token_logprobs_workspace_bytes(int(n_tokens), int(hidden_dim), int(vocab),
+                                                                 int(dtype_code)))
+
+
+# ------------------------------------------------------------------ the three calls
+def prefix_attn(q, k, v, cu_seqlens, max_seqlen: int, cache: Optional[Tuple] = None, softmax_scale: float = 0.0,
+                out=None, lse=None, return_lse: bool = False, workspace=None, device_status=None, stream=None):
+    """rpx_prefix_attn: causal GQA attention over packed prompts, writing the paged KV cache.
+
+    q [T, H_q, d], k/v [T, H_kv, d] device tensors; cu_seqlens int32 [B+1] on the device;
+    cache = (k_cache, v_cache, block_table) or None.  Returns out (and lse when asked).
+    """
+    torch = _torch()
+    lib = load_library()
+    desc = _desc(q, k, softmax_scale)
+    total = q.shape[0]
+    if out is None:
+        out = torch.empty((total, q.shape[1], q.shape[2]), dtype=q.dtype, device=q.device)
+    if lse is None and return_lse:
+        lse = torch.empty((total, q.shape[1]), dtype=torch.float32, device=q.device)
+    ws = _workspace(int(lib.rpx_prefix_attn_workspace_bytes(ctypes.byref(desc), total)), q.device, workspace)
+    cs = _cache_struct(cache) if cache is not None else None
+    rc = lib.rpx_prefix_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _tok_stride(q), _tok_stride(k),
+                             _tok_stride(v), _ptr(cu_seqlens), cu_seqlens.shape[0] - 1, total, int(max_seqlen),
+                             ctypes.byref(cs) if cs is not None else None, _ptr(out), _ptr(lse), _ptr(ws),
+                             ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_prefix_attn")
+    return (out, lse) if return_lse else out
+
+
+def suffix_attn(q, k, v, cu_seqlens_suffix, prefix_lens, max_suffix_len: int, max_prefix_len: int, cache: Tuple,
+                softmax_scale: float = 0.0, out=None, lse=None, return_lse: bool = False, workspace=None,
+                device_status=None, stream=None):
+    """rpx_suffix_attn: response queries over [cached prefix KV ; causal self]."""
+    torch = _torch()
+    lib = load_library()
+    desc = _desc(q, k, softmax_scale)
+    total = q.shape[0]
+    if out is None:
+        out = torch.empty((total, q.shape[1], q.shape[2]), dtype=q.dtype, device=q.device)
+    if lse is None and return_lse:
+        lse = torch.empty((total, q.shape[1]), dtype=torch.float32, device=q.device)
+    ws = _workspace(int(lib.rpx_suffix_attn_workspace_bytes(ctypes.byref(desc), total)), q.device, workspace)
+    cs = _cache_struct(cache)
+    rc = lib.rpx_suffix_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _tok_stride(q), _tok_stride(k),
+                             _tok_stride(v), _ptr(cu_seqlens_suffix), _ptr(prefix_lens),
+                             cu_seqlens_suffix.shape[0] - 1, total, int(max_suffix_len), int(max_prefix_len),
+                             ctypes.byref(cs), _ptr(out), _ptr(lse), _ptr(ws), ws.numel() * ws.element_size(),
+                             _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_suffix_attn")
+    return (out, lse) if return_lse else out
+
+
+def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_lse: bool = False, workspace=None,
+                   device_status=None, stream=None):
+    """rpx_token_logprobs: log p(target) per row from hidden [N, H] and W [V, H]; logits never stored."""
+    torch = _torch()
+    lib = load_library()
+    code = _dtype_code(hidden)
+    if _dtype_code(w_vocab) != code:
+        raise TypeError("hidden and w_vocab must share an element type")
+    if hidden.dim() != 2 or hidden.stride(1) != 1 or not w_vocab.is_contiguous():
+        raise ValueError("hidden must be [N, H] with contiguous rows and w_vocab contiguous [V, H]")
+    n, hdim = hidden.shape
+    vocab = w_vocab.shape[0]
+    if logprobs is None:
+        logprobs = torch.empty((n,), dtype=torch.float32, device=hidden.device)
+    if lse is None and return_lse:
+        lse = torch.empty((n,), dtype=torch.float32, device=hidden.device)
+    ws = _workspace(int(lib.rpx_token_logprobs_workspace_bytes(n, hdim, vocab, code)), hidden.device, workspace)
+    row_stride = hidden.stride(0) if n > 1 else hdim
+    rc = lib.rpx_token_logprobs(_ptr(hidden), row_stride, _ptr(w_vocab), _ptr(target_ids), n, hdim, vocab, code,
+                                _ptr(logprobs), _ptr(lse), _ptr(ws), ws.numel() * ws.element_size(),
+                                _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_token_logprobs")
+    return (logprobs, lse) if return_lse else logprobs
