@@ -40,6 +40,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define RPX_API __attribute__((visibility("default")))
+#else
+#define RPX_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -96,7 +102,7 @@ typedef struct {
  *   lse (nullable) float32 [total_tokens][num_q_heads]: ln sum_j exp(scale * q.k_j)
  *   max_seqlen: an upper bound on the longest sequence (sizes the grid).
  */
-rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+RPX_API rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
                              int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
                              const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens,
                              int32_t max_seqlen, const rpx_kv_cache_t* cache, void* out, float* lse,
@@ -113,7 +119,7 @@ rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const v
  *   cache: required, read-only here (response K/V are NOT appended; they have no later reader)
  *   max_suffix_len / max_prefix_len: upper bounds (grid sizing only).
  */
-rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+RPX_API rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
                              int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
                              const int32_t* cu_seqlens_suffix, const int32_t* prefix_lens, int32_t batch,
                              int64_t total_suffix_tokens, int32_t max_suffix_len, int32_t max_prefix_len,
@@ -132,23 +138,23 @@ rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const v
  * The kernel is position-agnostic: which (hidden row, next token) pairs form the prefix call and
  * which the suffix call is the caller's choice.
  */
-rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+RPX_API rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
                                 const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
                                 int32_t vocab, rpx_dtype_t dtype, float* logprobs, float* lse,
                                 void* workspace, size_t workspace_bytes, int32_t* device_status,
                                 void* cuda_stream);
 
 /* Workspace sizes in bytes for the calls above (pure host arithmetic; 0 is possible). */
-size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens);
-size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens);
-size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+RPX_API size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens);
+RPX_API size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens);
+RPX_API size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
                                           rpx_dtype_t dtype);
 
 /* Static string for a status code; never NULL. */
-const char* rpx_status_string(rpx_status_t status);
+RPX_API const char* rpx_status_string(rpx_status_t status);
 
 /* Library version: major * 10000 + minor * 100 + patch. */
-int32_t rpx_version(void);
+RPX_API int32_t rpx_version(void);
 
 #ifdef __cplusplus
 }

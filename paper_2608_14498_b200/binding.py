@@ -129,9 +129,13 @@ def _stream_ptr(stream) -> int:
 
 
 def _tok_stride(t) -> int:
-    if t.dim() != 3 or t.stride(2) != 1 or t.stride(1) != t.shape[2]:
+    if t.dim() != 3:
+        raise ValueError("expected a [tokens, heads, head_dim] tensor")
+    if t.shape[0] <= 1:
+        return t.shape[1] * t.shape[2]
+    if t.stride(2) != 1 or t.stride(1) != t.shape[2]:
         raise ValueError("expected a [tokens, heads, head_dim] tensor with contiguous heads")
-    return t.stride(0) if t.shape[0] > 1 else t.shape[1] * t.shape[2]
+    return t.stride(0)
 
 
 def _workspace(nbytes: int, device, workspace):

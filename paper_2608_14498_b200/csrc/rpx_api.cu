@@ -1,0 +1,216 @@
+// C-ABI front end: host-side validation, workspace carving, the fp32 -> bf16 pre-pass, and
+// dispatch to the sm_100a kernels.  Nothing here allocates device memory or synchronises.
+#include <cuda_bf16.h>
+
+#include "rpx_internal.h"
+
+namespace {
+
+using namespace rpx;
+
+constexpr size_t kWsAlign = 256;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+rpx_status_t check_attn_desc(const rpx_attn_desc_t* d) {
+    if (d == nullptr) return RPX_ERR_NULL;
+    if (d->dtype != RPX_BF16 && d->dtype != RPX_F32) return RPX_ERR_DTYPE;
+    if (d->head_dim != 64 && d->head_dim != 128) return RPX_ERR_SHAPE;
+    if (d->num_q_heads <= 0 || d->num_kv_heads <= 0 || d->num_q_heads % d->num_kv_heads != 0) return RPX_ERR_SHAPE;
+    return RPX_OK;
+}
+
+size_t attn_workspace(const rpx_attn_desc_t* d, int64_t tokens) {
+    if (d == nullptr || d->dtype != RPX_F32 || tokens <= 0) return 0;
+    const size_t qb = align_up(static_cast<size_t>(tokens) * d->num_q_heads * d->head_dim * 2, kWsAlign);
+    const size_t kb = align_up(static_cast<size_t>(tokens) * d->num_kv_heads * d->head_dim * 2, kWsAlign);
+    return qb + 2 * kb;
+}
+
+rpx_status_t check_cache(const rpx_kv_cache_t* c, int32_t batch) {
+    if (c->k_cache == nullptr || c->v_cache == nullptr || c->block_table == nullptr) return RPX_ERR_NULL;
+    if (c->block_size != 16 || c->num_blocks <= 0 || c->num_blocks > INT32_MAX) return RPX_ERR_SHAPE;
+    if (batch > 0 && c->block_table_stride <= 0) return RPX_ERR_SHAPE;
+    if (!aligned16(c->k_cache) || !aligned16(c->v_cache)) return RPX_ERR_ALIGN;
+    return RPX_OK;
+}
+
+// Shared body of the two attention entry points.  prefix_lens == NULL selects the prefix pass.
+rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                           int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const int32_t* cu_seqlens,
+                           const int32_t* prefix_lens, bool is_suffix, int32_t batch, int64_t total_tokens,
+                           int32_t max_q_len, int32_t max_prefix_len, const rpx_kv_cache_t* cache, void* out, float* lse,
+                           void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    if (rpx_status_t rc = check_attn_desc(desc)) return rc;
+    if (batch < 0 || total_tokens < 0 || max_q_len < 0 || max_prefix_len < 0) return RPX_ERR_SHAPE;
+    if (total_tokens >= INT32_MAX) return RPX_ERR_SHAPE;
+    if (is_suffix) {
+        if (cache == nullptr) return RPX_ERR_NULL;
+        if (batch > 0 && prefix_lens == nullptr) return RPX_ERR_NULL;
+    }
+    if (cache != nullptr)
+        if (rpx_status_t rc = check_cache(cache, batch)) return rc;
+    if (batch == 0 || total_tokens == 0 || max_q_len == 0) return RPX_OK;
+    if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || cu_seqlens == nullptr) return RPX_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return RPX_ERR_ALIGN;
+    const int64_t q_row = static_cast<int64_t>(desc->num_q_heads) * desc->head_dim;
+    const int64_t kv_row = static_cast<int64_t>(desc->num_kv_heads) * desc->head_dim;
+    if (q_tok_stride < q_row || k_tok_stride < kv_row || v_tok_stride < kv_row) return RPX_ERR_SHAPE;
+    if (q_tok_stride % 8 || k_tok_stride % 8 || v_tok_stride % 8) return RPX_ERR_ALIGN;
+    const size_t need = attn_workspace(desc, total_tokens);
+    if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return RPX_ERR_WORKSPACE;
+    if (need > 0 && !aligned16(workspace)) return RPX_ERR_ALIGN;
+    if (rpx_status_t rc = check_arch()) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    AttnArgs a;
+    a.num_q_heads = desc->num_q_heads;
+    a.num_kv_heads = desc->num_kv_heads;
+    a.head_dim = desc->head_dim;
+    a.softmax_scale = desc->softmax_scale;
+    a.q = q;
+    a.k = k;
+    a.v = v;
+    a.q_tok_stride = q_tok_stride;
+    a.k_tok_stride = k_tok_stride;
+    a.v_tok_stride = v_tok_stride;
+    if (desc->dtype == RPX_F32) {
+        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        const size_t qb = align_up(static_cast<size_t>(total_tokens) * q_row * 2, kWsAlign);
+        const size_t kb = align_up(static_cast<size_t>(total_tokens) * kv_row * 2, kWsAlign);
+        auto* qh = reinterpret_cast<__nv_bfloat16_raw*>(ws);
+        auto* kh = reinterpret_cast<__nv_bfloat16_raw*>(ws + qb);
+        auto* vh = reinterpret_cast<__nv_bfloat16_raw*>(ws + qb + kb);
+        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(q), q_tok_stride, qh, total_tokens, q_row, stream)) return rc;
+        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(k), k_tok_stride, kh, total_tokens, kv_row, stream)) return rc;
+        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(v), v_tok_stride, vh, total_tokens, kv_row, stream)) return rc;
+        a.q = qh;
+        a.k = kh;
+        a.v = vh;
+        a.q_tok_stride = q_row;
+        a.k_tok_stride = kv_row;
+        a.v_tok_stride = kv_row;
+    }
+    a.cu_seqlens = cu_seqlens;
+    a.prefix_lens = is_suffix ? prefix_lens : nullptr;
+    a.batch = batch;
+    a.total_tokens = total_tokens;
+    a.max_q_len = max_q_len;
+    a.max_prefix_len = max_prefix_len;
+    a.cache = cache;
+    a.out = out;
+    a.out_f32 = desc->dtype == RPX_F32;
+    a.lse = lse;
+    a.device_status = device_status;
+    a.stream = stream;
+    return launch_attention(a);
+}
+
+}  // namespace
+
+extern "C" {
+
+rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                             int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
+                             const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int32_t max_seqlen,
+                             const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens, nullptr, false, batch,
+                         total_tokens, max_seqlen, 0, cache, out, lse, workspace, workspace_bytes, device_status,
+                         cuda_stream);
+}
+
+rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                             int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
+                             const int32_t* cu_seqlens_suffix, const int32_t* prefix_lens, int32_t batch,
+                             int64_t total_suffix_tokens, int32_t max_suffix_len, int32_t max_prefix_len,
+                             const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens_suffix, prefix_lens, true,
+                         batch, total_suffix_tokens, max_suffix_len, max_prefix_len, cache, out, lse, workspace,
+                         workspace_bytes, device_status, cuda_stream);
+}
+
+size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens) {
+    return attn_workspace(desc, total_tokens);
+}
+
+size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens) {
+    return attn_workspace(desc, total_suffix_tokens);
+}
+
+size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype) {
+    if (n_tokens <= 0 || hidden_dim <= 0 || vocab <= 0) return 0;
+    size_t bytes = align_up(static_cast<size_t>(logprob_num_chunks(vocab)) * n_tokens * sizeof(float4), kWsAlign);
+    if (dtype == RPX_F32) {
+        bytes += align_up(static_cast<size_t>(n_tokens) * hidden_dim * 2, kWsAlign);
+        bytes += align_up(static_cast<size_t>(vocab) * hidden_dim * 2, kWsAlign);
+    }
+    return bytes;
+}
+
+rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                rpx_dtype_t dtype, float* logprobs, float* lse, void* workspace, size_t workspace_bytes,
+                                int32_t* device_status, void* cuda_stream) {
+    if (dtype != RPX_BF16 && dtype != RPX_F32) return RPX_ERR_DTYPE;
+    if (n_tokens < 0 || n_tokens >= INT32_MAX || hidden_dim <= 0 || vocab <= 0) return RPX_ERR_SHAPE;
+    if (hidden_dim % 8 != 0) return RPX_ERR_SHAPE;
+    if (n_tokens == 0) return RPX_OK;
+    if (hidden == nullptr || w_vocab == nullptr || target_ids == nullptr || logprobs == nullptr) return RPX_ERR_NULL;
+    if (hidden_row_stride < hidden_dim) return RPX_ERR_SHAPE;
+    if (hidden_row_stride % 8 != 0) return RPX_ERR_ALIGN;
+    if (!aligned16(hidden) || !aligned16(w_vocab)) return RPX_ERR_ALIGN;
+    const size_t need = rpx_token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype);
+    if (workspace == nullptr || workspace_bytes < need) return RPX_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return RPX_ERR_ALIGN;
+    if (rpx_status_t rc = check_arch()) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    LogprobArgs a;
+    a.partials = ws;
+    ws += align_up(static_cast<size_t>(logprob_num_chunks(vocab)) * n_tokens * sizeof(float4), kWsAlign);
+    a.hidden = hidden;
+    a.hidden_row_stride = hidden_row_stride;
+    a.w = w_vocab;
+    if (dtype == RPX_F32) {
+        auto* hh = reinterpret_cast<__nv_bfloat16_raw*>(ws);
+        ws += align_up(static_cast<size_t>(n_tokens) * hidden_dim * 2, kWsAlign);
+        auto* wh = reinterpret_cast<__nv_bfloat16_raw*>(ws);
+        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(hidden), hidden_row_stride, hh, n_tokens, hidden_dim, stream)) return rc;
+        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(w_vocab), hidden_dim, wh, vocab, hidden_dim, stream)) return rc;
+        a.hidden = hh;
+        a.hidden_row_stride = hidden_dim;
+        a.w = wh;
+    }
+    a.target_ids = target_ids;
+    a.n_tokens = n_tokens;
+    a.hidden_dim = hidden_dim;
+    a.vocab = vocab;
+    a.logprobs = logprobs;
+    a.lse = lse;
+    a.device_status = device_status;
+    a.stream = stream;
+    return launch_token_logprobs(a);
+}
+
+const char* rpx_status_string(rpx_status_t status) {
+    switch (status) {
+        case RPX_OK: return "ok";
+        case RPX_ERR_NULL: return "a required pointer is NULL";
+        case RPX_ERR_SHAPE: return "unsupported or inconsistent sizes";
+        case RPX_ERR_DTYPE: return "unknown element type";
+        case RPX_ERR_ALIGN: return "pointer or stride alignment";
+        case RPX_ERR_WORKSPACE: return "workspace missing or too small";
+        case RPX_ERR_ARCH: return "device is not compute capability 10.x (sm_100a kernels only)";
+        case RPX_ERR_CUDA: return "a CUDA call failed";
+        case RPX_ERR_DEVICE_DATA: return "out-of-range id in device data";
+        case RPX_ERR_TIMEOUT: return "a bounded kernel-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int32_t rpx_version(void) { return 100; }
+
+}  // extern "C"

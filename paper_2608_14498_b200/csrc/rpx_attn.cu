@@ -1,0 +1,565 @@
+// Varlen causal GQA flash attention for sm_100a, shared by the prefix pass (which also writes the
+// paged boundary-KV cache) and the suffix pass (which reads it back through the block table).
+//
+// One CTA owns two adjacent 128-row query tiles of one (sequence, query head) and walks the key
+// tiles (128 keys) that those rows may see: first the cached prefix tiles (suffix pass only,
+// unmasked except the last partial one), then the self tiles up to each query tile's diagonal.
+//   warps 0-3 : softmax of query tile 0   (thread = one row; TMEM lane = row)
+//   warps 4-7 : softmax of query tile 1
+//   warp  8   : TMA producer (Q once; K/V through a 3-slot ring; paged tiles = one TMA box per
+//               16-token page); it also stores the diagonal K/V tiles into the paged cache
+//   warp  9   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
+//               O_t += P_t V (P_t bf16 in swizzled smem, V as an MN-major operand)
+// The two query tiles alternate on the tensor core: while the softmax warps of one tile work on
+// S_t(j), the tensor core runs the other tile's PV(j-1) and QK(j).  Scores are kept in log2
+// units; O is rescaled lazily (only when a row's running max grows by more than 2^8).
+#include <math_constants.h>
+
+#include "rpx_internal.h"
+#include "rpx_ptx.cuh"
+
+namespace rpx {
+
+namespace {
+
+constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
+constexpr int kSlots = 3;
+constexpr int kThreads = 320;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;
+
+struct Ctl {
+    uint64_t q_full;
+    uint64_t kv_full[kSlots];
+    uint64_t kv_empty[kSlots];
+    uint64_t s_full[2];
+    uint64_t p_ready[2];
+    uint64_t pv_done[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t drain_flag;
+    uint32_t data_error;
+};
+
+template <int D>
+struct Layout {
+    static constexpr int kHalves = D / 64;               // 64-element (128-byte) column blocks
+    static constexpr int kHalfBytes = kTileK * 128;      // one [128 rows][64 bf16] swizzled block
+    static constexpr int kQBytes = kHalves * kHalfBytes; // one query tile
+    static constexpr int kKvBytes = kHalves * kHalfBytes;
+    static constexpr int kPBytes = 2 * kHalfBytes;       // [128 rows][128 keys] bf16
+    static constexpr int kQOff = 0;
+    static constexpr int kPOff = 2 * kQBytes;
+    static constexpr int kKvOff = kPOff + 2 * kPBytes;
+    static constexpr int kCtlOff = kKvOff + kSlots * kKvBytes;
+    static constexpr size_t kSmemBytes = 1024 + kCtlOff + sizeof(Ctl);
+};
+
+struct Params {
+    const int32_t* cu_seqlens;
+    const int32_t* prefix_lens;   // NULL: no cached prefix (prefix pass)
+    const int32_t* block_table;
+    int32_t block_table_stride;
+    int64_t num_blocks;
+    __nv_bfloat16* k_cache;       // used by the ragged-page paths
+    __nv_bfloat16* v_cache;
+    int32_t write_cache;          // prefix pass with a cache
+    int32_t batch, num_q_heads, num_kv_heads, group;
+    int32_t n_pairs;              // query tile pairs per sequence the grid covers
+    float scale_log2;
+    void* out;
+    int32_t out_f32;
+    float* lse;
+    int32_t* status;
+};
+
+// byte offset of 16-byte chunk `cc` (0..D/8-1) of row `r` inside a swizzled [128][D] tile
+__device__ __forceinline__ uint32_t swz_off(int r, int cc) {
+    return static_cast<uint32_t>((cc >> 3) * (kTileK * 128) + r * 128 + (((cc & 7) ^ (r & 7)) << 4));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
+            const __grid_constant__ CUtensorMap tmap_vc, const Params p) {
+    using L = Layout<D>;
+    // ---- which (pair, sequence, head) this CTA owns; late query tiles (most keys) launch first
+    const int32_t per_pair = p.batch * p.num_q_heads;
+    const int32_t pair = p.n_pairs - 1 - static_cast<int32_t>(blockIdx.x / per_pair);
+    const int32_t rem = static_cast<int32_t>(blockIdx.x % per_pair);
+    const int32_t seq = rem / p.num_q_heads;
+    const int32_t head = rem % p.num_q_heads;
+    const int32_t kv_head = head / p.group;
+    const int32_t tok0 = p.cu_seqlens[seq];
+    const int32_t len_q = p.cu_seqlens[seq + 1] - tok0;
+    const int32_t q0 = pair * 2 * kTileQ;
+    if (q0 >= len_q) return;  // uniform for the whole CTA, before any barrier or allocation
+    const int32_t len_p = p.prefix_lens != nullptr ? p.prefix_lens[seq] : 0;
+    const bool active1 = q0 + kTileQ < len_q;
+    const int32_t n_prefix_tiles = (len_p + kTileK - 1) / kTileK;
+    const int32_t n_tile[2] = {n_prefix_tiles + 2 * pair + 1, n_prefix_tiles + 2 * pair + 2};
+    const int32_t n_kv = active1 ? n_tile[1] : n_tile[0];
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + L::kCtlOff);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&ctl->q_full, 1);
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(&ctl->kv_full[s], 1);
+            mbar_init(&ctl->kv_empty[s], 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&ctl->s_full[t], 1);
+            mbar_init(&ctl->p_ready[t], 128);
+            mbar_init(&ctl->pv_done[t], 1);
+        }
+        mbar_init(&ctl->drain, 1);
+        ctl->abort_flag = 0;
+        ctl->drain_flag = 0;
+        ctl->data_error = 0;
+        fence_barrier_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(&ctl->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t tmem_s[2] = {tmem_base, tmem_base + 128};
+    const uint32_t tmem_o[2] = {tmem_base + 256, tmem_base + 384};
+
+    if (warp == 8) {
+        // =========================================================== producer warp
+        bool ok = true;
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_q);
+            tma_prefetch_desc(&tmap_k);
+            tma_prefetch_desc(&tmap_v);
+            mbar_arrive_expect_tx(&ctl->q_full, (active1 ? 2 : 1) * L::kQBytes);
+            for (int t = 0; t < (active1 ? 2 : 1); ++t)
+                for (int hf = 0; hf < L::kHalves; ++hf)
+                    tma_load_3d(smem + L::kQOff + t * L::kQBytes + hf * L::kHalfBytes, &tmap_q, &ctl->q_full,
+                                hf * 64, head, tok0 + q0 + t * kTileQ);
+        }
+        const bool owns_cache_write = p.write_cache != 0 && (head % p.group) == 0;
+        uint32_t n_loaded = 0;
+        for (int32_t j = 0; ok && j < n_kv; ++j) {
+            const bool from_cache = j < n_prefix_tiles;
+            const int32_t jt = from_cache ? j : j - n_prefix_tiles;  // tile index inside its key source
+            uint32_t slot_of[2];
+            for (int which = 0; which < 2; ++which, ++n_loaded) {  // 0 = K, 1 = V
+                const uint32_t slot = n_loaded % kSlots, phase = (n_loaded / kSlots) & 1u;
+                slot_of[which] = slot;
+                if (!mbar_wait(&ctl->kv_empty[slot], phase ^ 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                uint8_t* dst = smem + L::kKvOff + slot * L::kKvBytes;
+                if (!from_cache) {
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(&ctl->kv_full[slot], L::kKvBytes);
+                        for (int hf = 0; hf < L::kHalves; ++hf)
+                            tma_load_3d(dst + hf * L::kHalfBytes, which == 0 ? &tmap_k : &tmap_v, &ctl->kv_full[slot],
+                                        hf * 64, kv_head, tok0 + jt * kTileK);
+                    }
+                } else {
+                    // paged tile: whole 16-token pages by TMA; the ragged last page and the rows past
+                    // the prefix end by plain 16-byte copies / zero fill (a masked P of 0 must never
+                    // meet a non-finite stale V row)
+                    const int32_t rows_valid = min(kTileK, len_p - jt * kTileK);
+                    const int32_t full_pages = rows_valid / kPage;
+                    int32_t blk = 0;
+                    if (lane <= full_pages && lane < kTileK / kPage && jt * (kTileK / kPage) + lane < (len_p + kPage - 1) / kPage) {
+                        blk = p.block_table[static_cast<int64_t>(seq) * p.block_table_stride + jt * (kTileK / kPage) + lane];
+                        if (blk < 0 || blk >= p.num_blocks) {
+                            ctl->data_error = 1;
+                            blk = 0;
+                        }
+                    }
+                    if (full_pages < kTileK / kPage) {
+                        const int32_t blk_r = __shfl_sync(0xffffffffu, blk, full_pages);
+                        const __nv_bfloat16* src_pool = which == 0 ? p.k_cache : p.v_cache;
+                        const uint4* src = reinterpret_cast<const uint4*>(
+                            src_pool + (static_cast<int64_t>(blk_r) * p.num_kv_heads + kv_head) * kPage * D);
+                        const int32_t first_row = full_pages * kPage;
+                        const int32_t n_chunks = (kTileK - first_row) * (D / 8);
+                        for (int32_t i = lane; i < n_chunks; i += 32) {
+                            const int32_t r = first_row + i / (D / 8), cc = i % (D / 8);
+                            uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                            if (r < rows_valid) val = __ldg(src + (r - first_row) * (D / 8) + cc);
+                            *reinterpret_cast<uint4*>(dst + swz_off(r, cc)) = val;
+                        }
+                        fence_proxy_async_smem();
+                    }
+                    __syncwarp();
+                    for (int32_t pg = 0; pg < full_pages; ++pg) {
+                        const int32_t b = __shfl_sync(0xffffffffu, blk, pg);
+                        if (lane == 0) {
+                            if (pg == 0) mbar_arrive_expect_tx(&ctl->kv_full[slot], full_pages * kPage * D * 2);
+                            for (int hf = 0; hf < L::kHalves; ++hf)
+                                tma_load_4d(dst + hf * L::kHalfBytes + pg * (kPage * 128), which == 0 ? &tmap_kc : &tmap_vc,
+                                            &ctl->kv_full[slot], hf * 64, 0, kv_head, b);
+                        }
+                    }
+                    if (full_pages == 0 && lane == 0) mbar_arrive(&ctl->kv_full[slot]);
+                }
+                __syncwarp();
+            }
+            // ---- boundary-KV write: the two diagonal key tiles of this pair, one writer per KV head
+            if (ok && owns_cache_write && !from_cache && jt >= 2 * pair) {
+                for (int which = 0; which < 2 && ok; ++which) {
+                    const uint32_t idx = n_loaded - 2 + which;
+                    const uint32_t slot = slot_of[which];
+                    if (!mbar_wait(&ctl->kv_full[slot], (idx / kSlots) & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint8_t* src = smem + L::kKvOff + slot * L::kKvBytes;
+                    __nv_bfloat16* pool = which == 0 ? p.k_cache : p.v_cache;
+                    const int32_t rows_valid = min(kTileK, len_q - jt * kTileK);
+                    const int32_t n_pages = (rows_valid + kPage - 1) / kPage;
+                    int32_t blk = 0;
+                    if (lane < n_pages) {
+                        blk = p.block_table[static_cast<int64_t>(seq) * p.block_table_stride + jt * (kTileK / kPage) + lane];
+                        if (blk < 0 || blk >= p.num_blocks) {
+                            ctl->data_error = 1;
+                            blk = -1;
+                        }
+                    }
+                    for (int32_t pg = 0; pg < n_pages; ++pg) {
+                        const int32_t b = __shfl_sync(0xffffffffu, blk, pg);
+                        if (b < 0) continue;
+                        const int32_t rows = min(kPage, rows_valid - pg * kPage);
+                        if (rows == kPage) {
+                            if (lane == 0)
+                                for (int hf = 0; hf < L::kHalves; ++hf)
+                                    tma_store_4d(which == 0 ? &tmap_kc : &tmap_vc, src + hf * L::kHalfBytes + pg * (kPage * 128),
+                                                 hf * 64, 0, kv_head, b);
+                        } else {
+                            uint4* dstp = reinterpret_cast<uint4*>(
+                                pool + (static_cast<int64_t>(b) * p.num_kv_heads + kv_head) * kPage * D);
+                            for (int32_t i = lane; i < rows * (D / 8); i += 32) {
+                                const int32_t r = pg * kPage + i / (D / 8), cc = i % (D / 8);
+                                dstp[i] = *reinterpret_cast<const uint4*>(src + swz_off(r, cc));
+                            }
+                        }
+                    }
+                    if (lane == 0) {
+                        tma_store_commit();
+                        tma_store_wait_read();
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        if (!ok) {
+            // abort: give copies already in flight a moment to land before smem is released
+            const uint32_t first = n_loaded > kSlots ? n_loaded - kSlots : 0u;
+            for (uint32_t i = first; i < n_loaded; ++i)
+                mbar_wait(&ctl->kv_full[i % kSlots], (i / kSlots) & 1u, &ctl->drain_flag, 1000000ull);
+            mbar_wait(&ctl->q_full, 0, &ctl->drain_flag, 1000000ull);
+        }
+    } else if (warp == 9) {
+        // =========================================================== tcgen05 issuer (one thread)
+        if (elect_one()) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16(kTileQ, kTileK, false, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(kTileQ, D, false, true);
+            const uint32_t q_addr = smem_u32(smem + L::kQOff);
+            const uint32_t p_addr = smem_u32(smem + L::kPOff);
+            const uint32_t kv_addr = smem_u32(smem + L::kKvOff);
+            bool ok = true;
+
+            auto issue_qk = [&](int t, uint32_t k_slot) {
+                const uint32_t a0 = q_addr + t * L::kQBytes, b0 = kv_addr + k_slot * L::kKvBytes;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
+                    umma_bf16_ss(tmem_s[t], make_smem_desc_sw128(a0 + off, 16, 1024),
+                                 make_smem_desc_sw128(b0 + off, 16, 1024), idesc_qk, k != 0 ? 1u : 0u);
+                }
+                umma_commit(&ctl->s_full[t]);
+            };
+            auto issue_pv = [&](int t, uint32_t v_slot, bool accumulate) {
+                const uint32_t a0 = p_addr + t * L::kPBytes, b0 = kv_addr + v_slot * L::kKvBytes;
+#pragma unroll
+                for (int k = 0; k < kTileK / 16; ++k) {
+                    const uint32_t a_off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
+                    umma_bf16_ss(tmem_o[t], make_smem_desc_sw128(a0 + a_off, 16, 1024),
+                                 make_smem_desc_sw128(b0 + k * 2048, L::kHalfBytes, 1024), idesc_pv,
+                                 (accumulate || k != 0) ? 1u : 0u);
+                }
+                umma_commit(&ctl->pv_done[t]);
+            };
+
+            ok = mbar_wait(&ctl->q_full, 0, abort_flag);
+            if (ok) ok = mbar_wait(&ctl->kv_full[0], 0, abort_flag);  // K_0 is load 0
+            if (ok) {
+                tc_fence_after_sync();
+                issue_qk(0, 0);
+                if (active1) issue_qk(1, 0);
+                umma_commit(&ctl->kv_empty[0]);
+            }
+            for (int32_t j = 0; ok && j < n_kv; ++j) {
+                const uint32_t v_idx = 2 * j + 1, kn_idx = 2 * j + 2;
+                const uint32_t v_slot = v_idx % kSlots, kn_slot = kn_idx % kSlots;
+                bool have_v = false, have_kn = false;
+                for (int t = 0; t < 2 && ok; ++t) {
+                    if ((t == 1 && !active1) || j >= n_tile[t]) continue;
+                    if (!mbar_wait(&ctl->p_ready[t], j & 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    if (j + 1 < n_tile[t]) {
+                        if (!have_kn) {
+                            if (!mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after_sync();
+                            have_kn = true;
+                        }
+                        issue_qk(t, kn_slot);
+                    }
+                    if (!have_v) {
+                        if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        have_v = true;
+                    }
+                    issue_pv(t, v_slot, j != 0);
+                }
+                if (!ok) break;
+                if (have_kn) umma_commit(&ctl->kv_empty[kn_slot]);
+                umma_commit(&ctl->kv_empty[v_slot]);
+            }
+            if (!ok) {
+                umma_commit(&ctl->drain);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, 1000000ull);
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================================================== softmax warps
+        const int t = warp >> 2;
+        if (t == 0 || active1) {
+            const uint32_t quarter = warp & 3;
+            const int32_t row = quarter * 32 + lane;
+            const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
+            const uint32_t lane_addr = (quarter * 32u) << 16;
+            uint8_t* p_smem = smem + L::kPOff + t * L::kPBytes;
+            float run_max = -CUDART_INF_F, run_sum = 0.f;
+            bool ok = true;
+            for (int32_t j = 0; j < n_tile[t]; ++j) {
+                if (!mbar_wait(&ctl->s_full[t], j & 1, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                // ---- how many leading keys of this tile the row may see
+                int32_t n_vis;
+                if (j < n_prefix_tiles) {
+                    n_vis = min(kTileK, len_p - j * kTileK);
+                } else {
+                    const int32_t jt = j - n_prefix_tiles;
+                    n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
+                }
+                // ---- pass 1: row maximum (log2 units)
+                float cmax = -CUDART_INF_F;
+#pragma unroll 1
+                for (int c = 0; c < kTileK / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_s[t] + c * 32 + lane_addr, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float x = __uint_as_float(r[i]);
+                        cmax = fmaxf(cmax, (c * 32 + i < n_vis) ? x : -CUDART_INF_F);
+                    }
+                }
+                cmax *= p.scale_log2;  // scale > 0, so max commutes with the scaling
+                const bool grow = cmax > run_max + kRescaleThreshold;
+                const float new_max = grow ? cmax : run_max;
+                if (j > 0) {
+                    if (!mbar_wait(&ctl->pv_done[t], (j - 1) & 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    if (__any_sync(0xffffffffu, grow)) {
+                        const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
+#pragma unroll 1
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                            tmem_st32(tmem_o[t] + c * 32 + lane_addr, r);
+                        }
+                        tmem_st_wait();
+                        run_sum *= alpha;
+                    }
+                }
+                run_max = new_max;
+                // ---- pass 2: P = 2^(x - max) as bf16 into swizzled smem, row sum in fp32
+                const float neg_max = -run_max;
+                float part = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < kTileK / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_s[t] + c * 32 + lane_addr, r);
+                    tmem_ld_wait();
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float e0 = fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_max));
+                        float e1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_max));
+                        e0 = (c * 32 + i < n_vis) ? e0 : 0.f;
+                        e1 = (c * 32 + i + 1 < n_vis) ? e1 : 0.f;
+                        part += e0 + e1;
+                        packed[i >> 1] = pack_bf16x2(e0, e1);
+                    }
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        *reinterpret_cast<uint4*>(p_smem + swz_off(row, c * 4 + q4)) =
+                            make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
+                }
+                run_sum += part;
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&ctl->p_ready[t]);
+            }
+            // ---- epilogue: O / l -> global, LSE
+            if (ok && mbar_wait(&ctl->pv_done[t], (n_tile[t] - 1) & 1, abort_flag)) {
+                tc_fence_after_sync();
+                const bool row_valid = q_local < len_q;
+                const float inv = 1.f / run_sum;
+                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
+                    tmem_ld_wait();
+                    if (row_valid) {
+                        if (p.out_f32) {
+                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + out_row + c * 32);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                                                     __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + out_row + c * 32);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u)
+                                    w[u] = pack_bf16x2(__uint_as_float(r[8 * i + 2 * u]) * inv,
+                                                       __uint_as_float(r[8 * i + 2 * u + 1]) * inv);
+                                dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                    }
+                }
+                if (row_valid && p.lse != nullptr)
+                    p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && p.status != nullptr) {
+        if (ctl->abort_flag != 0u) atomicCAS(p.status, 0, RPX_ERR_TIMEOUT);
+        else if (ctl->data_error != 0u) atomicCAS(p.status, 0, RPX_ERR_DEVICE_DATA);
+    }
+}
+
+template <int D>
+rpx_status_t launch_attention_d(const AttnArgs& a) {
+    using L = Layout<D>;
+    CUtensorMap tq, tk, tv, tkc, tvc;
+    const uint64_t tokens = static_cast<uint64_t>(a.total_tokens);
+    {
+        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_q_heads), tokens};
+        const uint64_t strides[2] = {D * 2ull, static_cast<uint64_t>(a.q_tok_stride) * 2};
+        const uint32_t box[3] = {64, 1, kTileQ};
+        if (rpx_status_t rc = encode_tmap_bf16(&tq, a.q, 3, dims, strides, box)) return rc;
+    }
+    {
+        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_kv_heads), tokens};
+        const uint64_t ks[2] = {D * 2ull, static_cast<uint64_t>(a.k_tok_stride) * 2};
+        const uint64_t vs[2] = {D * 2ull, static_cast<uint64_t>(a.v_tok_stride) * 2};
+        const uint32_t box[3] = {64, 1, kTileK};
+        if (rpx_status_t rc = encode_tmap_bf16(&tk, a.k, 3, dims, ks, box)) return rc;
+        if (rpx_status_t rc = encode_tmap_bf16(&tv, a.v, 3, dims, vs, box)) return rc;
+    }
+    if (a.cache != nullptr) {
+        const uint64_t dims[4] = {D, kPage, static_cast<uint64_t>(a.num_kv_heads), static_cast<uint64_t>(a.cache->num_blocks)};
+        const uint64_t strides[3] = {D * 2ull, kPage * D * 2ull, static_cast<uint64_t>(a.num_kv_heads) * kPage * D * 2ull};
+        const uint32_t box[4] = {64, kPage, 1, 1};
+        if (rpx_status_t rc = encode_tmap_bf16(&tkc, a.cache->k_cache, 4, dims, strides, box)) return rc;
+        if (rpx_status_t rc = encode_tmap_bf16(&tvc, a.cache->v_cache, 4, dims, strides, box)) return rc;
+    } else {
+        tkc = tk;  // never dereferenced without a cache
+        tvc = tv;
+    }
+    Params p;
+    p.cu_seqlens = a.cu_seqlens;
+    p.prefix_lens = a.prefix_lens;
+    p.block_table = a.cache ? a.cache->block_table : nullptr;
+    p.block_table_stride = a.cache ? a.cache->block_table_stride : 0;
+    p.num_blocks = a.cache ? a.cache->num_blocks : 0;
+    p.k_cache = a.cache ? static_cast<__nv_bfloat16*>(a.cache->k_cache) : nullptr;
+    p.v_cache = a.cache ? static_cast<__nv_bfloat16*>(a.cache->v_cache) : nullptr;
+    p.write_cache = (a.cache != nullptr && a.prefix_lens == nullptr) ? 1 : 0;
+    p.batch = a.batch;
+    p.num_q_heads = a.num_q_heads;
+    p.num_kv_heads = a.num_kv_heads;
+    p.group = a.num_q_heads / a.num_kv_heads;
+    p.n_pairs = (a.max_q_len + 2 * kTileQ - 1) / (2 * kTileQ);
+    const float scale = a.softmax_scale > 0.f ? a.softmax_scale : 1.0f / sqrtf(static_cast<float>(D));
+    p.scale_log2 = scale * kLog2e;
+    p.out = a.out;
+    p.out_f32 = a.out_f32 ? 1 : 0;
+    p.lse = a.lse;
+    p.status = a.device_status;
+    const int64_t grid = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
+    if (grid <= 0) return RPX_OK;
+    if (grid > INT32_MAX) return RPX_ERR_SHAPE;
+    if (cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(L::kSmemBytes)) != cudaSuccess)
+        return RPX_ERR_CUDA;
+    attn_kernel<D><<<static_cast<unsigned>(grid), kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tkc, tvc, p);
+    return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
+}
+
+}  // namespace
+
+rpx_status_t launch_attention(const AttnArgs& a) {
+    if (a.total_tokens == 0 || a.batch == 0 || a.max_q_len == 0) return RPX_OK;
+    if (a.head_dim == 128) return launch_attention_d<128>(a);
+    if (a.head_dim == 64) return launch_attention_d<64>(a);
+    return RPX_ERR_SHAPE;
+}
+
+}  // namespace rpx

@@ -1,0 +1,87 @@
+// Host utilities: tensor-map encoding through the runtime's driver entry point lookup, device
+// queries, and the fp32 -> bf16 pre-pass used for RPX_F32 inputs.
+#include <cuda_bf16.h>
+
+#include <mutex>
+
+#include "rpx_internal.h"
+
+namespace rpx {
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+__global__ void cast_f32_bf16_kernel(const float* __restrict__ src, int64_t src_row_stride,
+                                     __nv_bfloat16* __restrict__ dst, int64_t rows, int64_t cols) {
+    const int64_t total = rows * cols;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / cols, c = i - r * cols;
+        dst[i] = __float2bfloat16_rn(src[r * src_row_stride + c]);
+    }
+}
+
+}  // namespace
+
+rpx_status_t encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                              const uint64_t* strides_bytes, const uint32_t* box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return RPX_ERR_CUDA;
+    cuuint64_t gdim[5], gstride[4];
+    cuuint32_t bdim[5], estride[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bdim[i] = box[i];
+        estride[i] = 1;
+        if (i + 1 < rank) gstride[i] = strides_bytes[i];
+    }
+    const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+                           gdim, gstride, bdim, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? RPX_OK : RPX_ERR_CUDA;
+}
+
+int sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return n;
+}
+
+rpx_status_t check_arch() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RPX_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RPX_ERR_CUDA;
+    return major == 10 ? RPX_OK : RPX_ERR_ARCH;
+}
+
+rpx_status_t launch_cast_f32_bf16(const float* src, int64_t src_row_stride, __nv_bfloat16_raw* dst, int64_t rows,
+                                  int64_t cols, cudaStream_t stream) {
+    const int64_t total = rows * cols;
+    if (total == 0) return RPX_OK;
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    const int64_t cap = static_cast<int64_t>(sm_count() > 0 ? sm_count() : 148) * 16;
+    if (blocks > cap) blocks = cap;
+    cast_f32_bf16_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+        src, src_row_stride, reinterpret_cast<__nv_bfloat16*>(dst), rows, cols);
+    return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
+}
+
+}  // namespace rpx

@@ -1,0 +1,64 @@
+// Host-side declarations shared by the C-ABI front end and the kernel launchers.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "rpx.h"
+
+namespace rpx {
+
+// Encodes a tiled bf16 tensor map with 128-byte swizzle (inner box extent must be 64 elements).
+// dims/strides innermost first; strides_bytes has rank-1 entries (the innermost is contiguous).
+// cuTensorMapEncodeTiled is looked up through the runtime, so libcuda is not a link dependency.
+rpx_status_t encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                              const uint64_t* strides_bytes, const uint32_t* box);
+
+int sm_count();                 // multiprocessors of the current device (cached per device)
+rpx_status_t check_arch();      // RPX_OK on compute capability 10.x
+
+// f32 -> bf16 (round to nearest even) of `rows` rows of `cols` contiguous elements.
+rpx_status_t launch_cast_f32_bf16(const float* src, int64_t src_row_stride, __nv_bfloat16_raw* dst, int64_t rows,
+                                  int64_t cols, cudaStream_t stream);
+
+struct AttnArgs {
+    int32_t num_q_heads, num_kv_heads, head_dim;
+    float softmax_scale;
+    const void *q, *k, *v;             // bf16
+    int64_t q_tok_stride, k_tok_stride, v_tok_stride;
+    const int32_t* cu_seqlens;         // query/self-key packing
+    const int32_t* prefix_lens;        // NULL for the prefix pass
+    int32_t batch;
+    int64_t total_tokens;
+    int32_t max_q_len, max_prefix_len;
+    const rpx_kv_cache_t* cache;       // prefix pass: written (nullable); suffix pass: read
+    void* out;
+    bool out_f32;
+    float* lse;
+    int32_t* device_status;
+    cudaStream_t stream;
+};
+rpx_status_t launch_attention(const AttnArgs& a);
+
+struct LogprobArgs {
+    const void* hidden;   // bf16 [n][hidden_row_stride]
+    int64_t hidden_row_stride;
+    const void* w;        // bf16 [vocab][hidden_dim]
+    const int32_t* target_ids;
+    int64_t n_tokens;
+    int32_t hidden_dim, vocab;
+    float* logprobs;
+    float* lse;
+    void* partials;       // float4 [logprob_num_chunks(vocab)][n_tokens]
+    int32_t* device_status;
+    cudaStream_t stream;
+};
+int32_t logprob_num_chunks(int32_t vocab);
+rpx_status_t launch_token_logprobs(const LogprobArgs& a);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace rpx

@@ -1,0 +1,343 @@
+// Fused LM-head log-probabilities for sm_100a.
+//
+//   logprob[n] = z[n, target[n]] - ln sum_v exp(z[n, v]),   z = hidden . W_vocab^T  (never stored)
+//
+// One persistent CTA per SM.  A work item is (row tile of 128 rows, chunk of kTilesPerChunk vocab
+// tiles of 256 columns): the CTA sweeps the chunk tile by tile; each tile is a TMA-fed tcgen05
+// GEMM over the hidden dimension into one of two 128x256 fp32 TMEM accumulators, and while the
+// tensor core fills one accumulator the four epilogue warps fold the other into a running
+// (max, sum-exp, target-logit) per row.  One partial per (chunk, row) goes to the workspace; a
+// small second kernel merges the partials.  Items are ordered so that the CTAs resident at any
+// moment cover a few vocab chunks times many row tiles: every W tile is pulled from HBM once per
+// wave and shared through L2, and the wave's hidden rows stay L2-resident across the chunk.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
+#include <math_constants.h>
+
+#include "rpx_internal.h"
+#include "rpx_ptx.cuh"
+
+namespace rpx {
+
+namespace {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
+constexpr int kTilesPerChunk = 16;
+constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct Ctl {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t drain_flag;
+};
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * (kABytes + kBBytes) + sizeof(Ctl);
+
+struct Params {
+    int64_t n_rows;
+    int32_t vocab;
+    int32_t k_blocks;      // ceil(hidden_dim / 64)
+    int32_t n_row_tiles;
+    int32_t n_vocab_tiles;
+    int32_t n_chunks;
+    int32_t group_width;   // vocab chunks in flight side by side
+    int32_t total_items;
+    const int32_t* target_ids;
+    float4* partials;      // [n_chunks][n_rows]: (max in log2 units, sum of 2^(x-max), target logit, 0)
+    int32_t* status;
+};
+
+struct Item {
+    int32_t m_tile, chunk, tile_begin, tile_end;
+};
+
+__device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
+    const int32_t per_group = p.n_row_tiles * p.group_width;
+    const int32_t cg = idx / per_group;
+    const int32_t rem = idx - cg * per_group;
+    const int32_t first = cg * p.group_width;
+    const int32_t width = min(p.group_width, p.n_chunks - first);
+    Item it;
+    it.m_tile = rem / width;
+    it.chunk = first + rem % width;
+    it.tile_begin = it.chunk * kTilesPerChunk;
+    it.tile_end = min(it.tile_begin + kTilesPerChunk, p.n_vocab_tiles);
+    return it;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
+                       const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem_a = smem;
+    uint8_t* smem_b = smem + kStages * kABytes;
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + kStages * (kABytes + kBBytes));
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&ctl->tmem_full[a], 1);
+            mbar_init(&ctl->tmem_empty[a], 128);
+        }
+        mbar_init(&ctl->drain, 1);
+        ctl->abort_flag = 0;
+        ctl->drain_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmap_hidden);
+        tma_prefetch_desc(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(&ctl->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one thread)
+        if (elect_one()) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
+                const Item item = decode_item(p, idx);
+                for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t) {
+                    for (int32_t kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                        const uint32_t stage = it % kStages, phase = (it / kStages) & 1u;
+                        if (!mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(&ctl->full[stage], kABytes + kBBytes);
+                        tma_load_2d(smem_a + stage * kABytes, &tmap_hidden, &ctl->full[stage], kb * kBK,
+                                    item.m_tile * kBM);
+                        tma_load_2d(smem_b + stage * kBBytes, &tmap_w, &ctl->full[stage], kb * kBK, t * kBN);
+                    }
+                }
+            }
+            if (!ok) {
+                // abort: let the copies already in flight land before the CTA's smem goes away
+                const uint32_t first = it > kStages ? it - kStages : 0u;
+                for (uint32_t j = first; j < it; ++j)
+                    mbar_wait(&ctl->full[j % kStages], (j / kStages) & 1u, &ctl->drain_flag, 1000000ull);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one thread)
+        if (elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, false, false);
+            uint32_t it = 0, tile_count = 0;
+            bool ok = true;
+            for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
+                const Item item = decode_item(p, idx);
+                for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
+                    const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + acc * kBN;
+                    for (int32_t kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                        const uint32_t stage = it % kStages, phase = (it / kStages) & 1u;
+                        if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = smem_u32(smem_a + stage * kABytes);
+                        const uint32_t b_addr = smem_u32(smem_b + stage * kBBytes);
+#pragma unroll
+                        for (int k = 0; k < kBK / 16; ++k) {
+                            umma_bf16_ss(d_tmem, make_smem_desc_sw128(a_addr + k * 32, 16, 1024),
+                                         make_smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc,
+                                         (kb | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit(&ctl->empty[stage]);
+                    }
+                    if (ok) umma_commit(&ctl->tmem_full[acc]);
+                }
+            }
+            if (!ok) {
+                umma_commit(&ctl->drain);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, 1000000ull);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (128 threads)
+        const uint32_t quarter = warp & 3;
+        const int32_t row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (quarter * 32u) << 16;
+        uint32_t tile_count = 0;
+        bool ok = true;
+        for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
+            const Item item = decode_item(p, idx);
+            const int64_t row = static_cast<int64_t>(item.m_tile) * kBM + row_in_tile;
+            const bool valid = row < p.n_rows;
+            const int32_t target = valid ? __ldg(p.target_ids + row) : -1;
+            float run_max = -CUDART_INF_F, run_sum = 0.f, target_logit = 0.f;
+            for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
+                const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const int32_t n0 = t * kBN;
+#pragma unroll 1
+                for (int c = 0; c < kBN / 32; ++c) {
+                    const int32_t col0 = n0 + c * 32;
+                    if (col0 >= p.vocab) break;
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + acc * kBN + c * 32 + lane_addr, r);
+                    tmem_ld_wait();
+                    float x[32];
+                    float cmax = -CUDART_INF_F;
+                    if (col0 + 32 <= p.vocab) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            x[i] = __uint_as_float(r[i]) * kLog2e;
+                            cmax = fmaxf(cmax, x[i]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            x[i] = (col0 + i < p.vocab) ? __uint_as_float(r[i]) * kLog2e : -CUDART_INF_F;
+                            cmax = fmaxf(cmax, x[i]);
+                        }
+                    }
+                    const uint32_t tl = static_cast<uint32_t>(target - col0);
+                    if (tl < 32u) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (tl == static_cast<uint32_t>(i)) target_logit = __uint_as_float(r[i]);
+                    }
+                    const float new_max = fmaxf(run_max, cmax);
+                    run_sum *= fast_exp2(run_max - new_max);
+                    float part = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) part += fast_exp2(x[i] - new_max);
+                    run_sum += part;
+                    run_max = new_max;
+                }
+                tc_fence_before_sync();
+                mbar_arrive(&ctl->tmem_empty[acc]);
+            }
+            if (ok && valid)
+                p.partials[static_cast<int64_t>(item.chunk) * p.n_rows + row] =
+                    make_float4(run_max, run_sum, target_logit, 0.f);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && ctl->abort_flag != 0u && p.status != nullptr) atomicCAS(p.status, 0, RPX_ERR_TIMEOUT);
+}
+
+__global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int32_t n_chunks, int64_t n_rows,
+                                       const int32_t* __restrict__ target_ids, int32_t vocab,
+                                       float* __restrict__ logprobs, float* __restrict__ lse, int32_t* status) {
+    const int64_t row = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
+    if (row >= n_rows) return;
+    float gmax = -CUDART_INF_F;
+    for (int32_t c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, partials[static_cast<int64_t>(c) * n_rows + row].x);
+    float sum = 0.f, zt = 0.f;
+    for (int32_t c = 0; c < n_chunks; ++c) {
+        const float4 v = partials[static_cast<int64_t>(c) * n_rows + row];
+        sum += v.y * exp2f(v.x - gmax);
+        zt += v.z;
+    }
+    const float l = (gmax + log2f(sum)) * kLn2;
+    const int32_t t = target_ids[row];
+    float lp;
+    if (t < 0 || t >= vocab) {
+        lp = CUDART_NAN_F;
+        if (status != nullptr) atomicCAS(status, 0, RPX_ERR_DEVICE_DATA);
+    } else {
+        lp = zt - l;
+    }
+    logprobs[row] = lp;
+    if (lse != nullptr) lse[row] = l;
+}
+
+}  // namespace
+
+int32_t logprob_num_chunks(int32_t vocab) {
+    const int32_t tiles = (vocab + kBN - 1) / kBN;
+    return (tiles + kTilesPerChunk - 1) / kTilesPerChunk;
+}
+
+rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
+    if (a.n_tokens == 0) return RPX_OK;
+    CUtensorMap tmap_h, tmap_w;
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(a.hidden_dim), static_cast<uint64_t>(a.n_tokens)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a.hidden_row_stride) * 2};
+        const uint32_t box[2] = {kBK, kBM};
+        if (rpx_status_t rc = encode_tmap_bf16(&tmap_h, a.hidden, 2, dims, strides, box)) return rc;
+    }
+    {
+        const uint64_t dims[2] = {static_cast<uint64_t>(a.hidden_dim), static_cast<uint64_t>(a.vocab)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a.hidden_dim) * 2};
+        const uint32_t box[2] = {kBK, kBN};
+        if (rpx_status_t rc = encode_tmap_bf16(&tmap_w, a.w, 2, dims, strides, box)) return rc;
+    }
+    Params p;
+    p.n_rows = a.n_tokens;
+    p.vocab = a.vocab;
+    p.k_blocks = (a.hidden_dim + kBK - 1) / kBK;
+    p.n_row_tiles = static_cast<int32_t>((a.n_tokens + kBM - 1) / kBM);
+    p.n_vocab_tiles = (a.vocab + kBN - 1) / kBN;
+    p.n_chunks = logprob_num_chunks(a.vocab);
+    const int64_t total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
+    if (total > INT32_MAX) return RPX_ERR_SHAPE;
+    p.total_items = static_cast<int32_t>(total);
+    const int sms = sm_count();
+    if (sms <= 0) return RPX_ERR_CUDA;
+    const int grid = static_cast<int>(total < sms ? total : sms);
+    p.group_width = (grid % 4 == 0) ? 4 : (grid % 2 == 0 ? 2 : 1);
+    p.target_ids = a.target_ids;
+    p.partials = static_cast<float4*>(a.partials);
+    p.status = a.device_status;
+
+    static bool attr_set = false;  // idempotent; a race only repeats the call
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(lm_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSmemBytes)) != cudaSuccess)
+            return RPX_ERR_CUDA;
+        attr_set = true;
+    }
+    lm_head_partial_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w, p);
+    if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    const int cthreads = 256;
+    const unsigned cblocks = static_cast<unsigned>((a.n_tokens + cthreads - 1) / cthreads);
+    lm_head_combine_kernel<<<cblocks, cthreads, 0, a.stream>>>(p.partials, p.n_chunks, a.n_tokens, a.target_ids,
+                                                               a.vocab, a.logprobs, a.lse, a.device_status);
+    return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
+}
+
+}  // namespace rpx

@@ -1,0 +1,108 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every declared symbol,
+and rejects host-checkable mistakes before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__  # noqa: F401  (builds librpx.so on import of build())
+from paper_2608_14498_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_14498_b200 import build
+
+    build.build()
+    return B.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "rpx.h")).read()
+    declared = re.findall(r"RPX_API[^;(]*?\b(rpx_\w+)\s*\(", header)
+    assert sorted(declared) == sorted(B.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert B.version() == 100
+    seen = set()
+    for code in range(0, -10, -1):
+        s = B.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 10
+    assert B.status_string(-99) == "unknown status"
+
+
+def test_workspace_arithmetic(lib):
+    assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 32768) == 0
+    need = B.prefix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 256)
+    assert need == 256 * 4 * 64 * 2 + 2 * 256 * 2 * 64 * 2
+    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 32 * 8 * 64 * 2
+    # 152064 columns = 594 tiles of 256 = 38 chunks of 16 tiles; one float4 per (chunk, row)
+    assert B.token_logprobs_workspace_bytes(34816, 3584, 152064, B.RPX_BF16) == 38 * 34816 * 16
+    f32 = B.token_logprobs_workspace_bytes(288, 256, 4096, B.RPX_F32)
+    assert f32 == 1 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
+    assert B.token_logprobs_workspace_bytes(0, 256, 4096, B.RPX_BF16) == 0
+
+
+def _attn_call(lib, desc, q=0x1000, k=0x1000, v=0x1000, strides=(512, 256, 256), cu=0x1000, batch=1, total=16,
+               max_len=16, cache=None, out=0x1000, ws=None, ws_bytes=0):
+    return lib.rpx_prefix_attn(ctypes.byref(desc), q, k, v, strides[0], strides[1], strides[2], cu, batch, total, max_len,
+                               cache, out, None, ws, ws_bytes, None, None)
+
+
+def test_attention_rejects_bad_arguments_before_any_launch(lib):
+    good = B.AttnDesc(4, 2, 128, 0.0, B.RPX_BF16)
+    assert lib.rpx_prefix_attn(None, 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, 1, 16, 16, None, 0x1000, None, None,
+                               0, None, None) == -1
+    assert _attn_call(lib, B.AttnDesc(4, 3, 128, 0.0, B.RPX_BF16)) == -2  # heads not divisible
+    assert _attn_call(lib, B.AttnDesc(4, 2, 96, 0.0, B.RPX_BF16)) == -2  # head_dim
+    assert _attn_call(lib, B.AttnDesc(4, 2, 128, 0.0, 7)) == -3  # dtype
+    assert _attn_call(lib, good, q=None) == -1
+    assert _attn_call(lib, good, q=0x1008) == -4
+    assert _attn_call(lib, good, strides=(516, 256, 256)) == -4
+    assert _attn_call(lib, good, strides=(256, 256, 256)) == -2  # token stride shorter than a row
+    assert _attn_call(lib, good, total=-1) == -2
+    assert _attn_call(lib, B.AttnDesc(4, 2, 128, 0.0, B.RPX_F32), ws=None, ws_bytes=0) == -5
+    # legal no-ops need neither pointers nor a device
+    assert _attn_call(lib, good, q=None, batch=0, total=0) == 0
+    assert _attn_call(lib, good, q=None, total=0) == 0
+    bad_cache = B.KvCache(0x1000, 0x1000, 8, 32, 0x1000, 4)
+    assert _attn_call(lib, good, cache=ctypes.byref(bad_cache)) == -2  # block size must be 16
+    null_cache = B.KvCache(None, 0x1000, 8, 16, 0x1000, 4)
+    assert _attn_call(lib, good, cache=ctypes.byref(null_cache)) == -1
+    # the suffix pass needs a cache and prefix lengths
+    rc = lib.rpx_suffix_attn(ctypes.byref(good), 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, 0x1000, 1, 16, 16, 64,
+                             None, 0x1000, None, None, 0, None, None)
+    assert rc == -1
+
+
+def test_logprobs_rejects_bad_arguments_before_any_launch(lib):
+    def call(hidden=0x1000, stride=256, w=0x1000, ids=0x1000, n=8, h=256, v=4096, dt=B.RPX_BF16, lp=0x1000, ws=0x1000,
+             ws_bytes=1 << 30):
+        return lib.rpx_token_logprobs(hidden, stride, w, ids, n, h, v, dt, lp, None, ws, ws_bytes, None, None)
+
+    assert call(dt=5) == -3
+    assert call(h=100) == -2
+    assert call(v=0) == -2
+    assert call(hidden=None) == -1
+    assert call(lp=None) == -1
+    assert call(stride=128) == -2
+    assert call(stride=260) == -4
+    assert call(w=0x1004) == -4
+    assert call(ws=None) == -5
+    assert call(ws_bytes=16) == -5
+    assert call(n=0, hidden=None) == 0
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "_LIB_PATH", str(tmp_path / "librpx.so"))
+    with pytest.raises(FileNotFoundError):
+        B.load_library()
