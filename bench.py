@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the prefix+suffix scoring hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C2]
+
+One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
+boundary-KV write), prefix log-probs, suffix attention over the cached KV, suffix log-probs.
+Metric: scored tokens/s (every token of every sequence gets a log-prob) and TFLOP/s.
+
+`value`     inputs already resident in HBM, timed with CUDA events on the launching stream.
+`e2e`       the same pass from pinned HOST tensors through ScoringSession.score_from_host:
+            host->device copies of the step's inputs and the device->host read of the log-probs
+            are inside the timed region (W_vocab is a model weight and stays resident).
+`roofline`  the dominant kernel (the fused LM-head kernel on the prompt rows): algorithmic FLOPs
+            / its CUDA-event duration, against the measured dense-bf16 peak of this machine.
+`cpu_baseline`  the fp64 oracle, as it stands, on a bounded sample of the same workload.
+`--impl reference` times that oracle alone (rank 0 only).
+
+N > 1 (torchrun): every rank scores its own batch of the same shape (sequences are independent,
+W_vocab replicated, no data-path collective) => weak scaling; time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_14498_b200 import workloads as wk  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (read + write) of one LM-head partial-kernel launch on the bench workload, scaled from
+# an ncu capture of a smaller launch of the same kernel; see profiles/.  None until captured.
+LM_HEAD_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def flop_counts(wl):
+    cfg = wl.cfg
+    p = wl.prompt_lens.astype(np.float64)
+    r = wl.response_lens.astype(np.float64)
+    d, hq = cfg.head_dim, cfg.num_q_heads
+    return {
+        "prefix_attn": float((2.0 * d * hq * p * (p + 1)).sum()),
+        "suffix_attn": float((4.0 * d * hq * (r * p + r * (r + 1) / 2)).sum()),
+        "lm_prefix": 2.0 * wl.n_prefix * cfg.hidden * cfg.vocab,
+        "lm_suffix": 2.0 * wl.n_suffix * cfg.hidden * cfg.vocab,
+    }
+
+
+def host_batch(wl, torch, pin=True):
+    """Pinned host tensors of one batch, laid out as the library takes them."""
+    from paper_2608_14498_b200.pipeline import Batch
+
+    def t(a):
+        if a.dtype == np.uint16:
+            x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+        else:
+            x = torch.from_numpy(a)
+        return x.pin_memory() if pin else x
+
+    pre, suf = wl.prefix_rows(), wl.suffix_rows()
+    return Batch(
+        t(wl.q[pre]), t(wl.k[pre]), t(wl.v[pre]), t(wl.q[suf]), t(wl.k[suf]), t(wl.v[suf]),
+        t(wl.cu_prefix), t(wl.cu_suffix), t(wl.prompt_lens), t(wl.block_table),
+        t(wl.hidden[pre]), t(wl.ids[pre]), t(wl.hidden[suf]), t(wl.ids[suf]),
+        int(wl.prompt_lens.max()), int(wl.response_lens.max()))
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+        self.marks = []
+
+    def mark(self):
+        self.tmp.flush()
+        self.marks.append(os.path.getsize(self.tmp.name))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        with open(self.tmp.name) as fh:
+            data = fh.read()
+        os.unlink(self.tmp.name)
+        lo = self.marks[0] if self.marks else 0
+        hi = self.marks[1] if len(self.marks) > 1 else len(data)
+        rows = [ln.split(",") for ln in data[lo:hi].splitlines() if ln.count(",") >= 7]
+        all_rows = [ln.split(",") for ln in data.splitlines() if ln.count(",") >= 7]
+        rows = rows or all_rows
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm, reasons = [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.strip().lower() == "active":
+                    reasons.add(name)
+        try:
+            sm_max = float(rows[0][1])
+        except ValueError:
+            sm_max = None
+        power = [float(r[2]) for r in rows if r[2].strip().replace(".", "", 1).isdigit()]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": sm_max, "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+def oracle_sample(wl, n_tokens: int, seed: int):
+    """Scores `n_tokens` sampled tokens with the oracle (all query heads + the log-prob row).
+    Returns seconds."""
+    import oracle
+
+    cfg = wl.cfg
+    rng = np.random.default_rng(seed)
+    tok = np.sort(rng.choice(wl.n_tokens, size=n_tokens, replace=False)).astype(np.int64)
+    seq = np.searchsorted(wl.cu_full, tok, side="right") - 1
+    pos = tok - wl.cu_full[seq]
+    rows = np.stack([np.repeat(seq, cfg.num_q_heads), np.repeat(pos, cfg.num_q_heads),
+                     np.tile(np.arange(cfg.num_q_heads), n_tokens)], axis=1).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.attn_rows(wl.q, wl.k, wl.v, wl.cu_full, rows)
+    oracle.logprob_rows(wl.hidden, wl.w, wl.ids, tok)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    import oracle
+
+    oracle.build()
+    cfg = wk.CONFIGS[args.config]
+    wl = wk.make_workload(cfg, seed=0)
+    n = args.ref_tokens
+    for w in range(args.warmup):
+        oracle_sample(wl, n, 1000 + w)
+    t = 0.0
+    for s in range(args.steps):
+        t += oracle_sample(wl, n, s)
+    value = args.steps * n / t
+    cores = oracle.num_threads()
+    sample = f"{n} tokens per step drawn uniformly from the batch: {cfg.num_q_heads} attention rows + 1 log-prob row each, fp64"
+    line = {
+        "impl": "reference", "metric": "scored_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_14498_b200 as rpx
+    from paper_2608_14498_b200.pipeline import KERNELS_PER_SCORE, Batch, ScoringSession
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
+    rpx.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    cfg = wk.CONFIGS[args.config]
+    wl = wk.make_workload(cfg, seed=rank)
+    flops = flop_counts(wl)
+    hb = host_batch(wl, torch)
+    db = Batch(*[x.to(dev) for x in hb.tensors()], hb.max_prefix_len, hb.max_suffix_len)
+    w_dev = torch.from_numpy(wl.w.view(np.int16)).view(torch.bfloat16).to(dev) if wl.w.dtype == np.uint16 \
+        else torch.from_numpy(wl.w).to(dev)
+    sess = ScoringSession(w_dev, wl.num_blocks, cfg.num_kv_heads, cfg.head_dim)
+    lp_p_host = torch.empty(wl.n_prefix, dtype=torch.float32).pin_memory()
+    lp_s_host = torch.empty(wl.n_suffix, dtype=torch.float32).pin_memory()
+
+    for _ in range(max(args.warmup, 3)):
+        sess.score(db)
+    torch.cuda.synchronize()
+    sess.check_status()
+
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(local_rank).uuid)
+        gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id) if rank == 0 else None
+    time.sleep(0.3)
+
+    # ---------------- device-resident timing: events around every call of every step
+    names = ["prefix_attn", "lm_prefix", "suffix_attn", "lm_suffix"]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.mark()
+    for s in range(args.steps):
+        sess.score(db, events=ev[s])
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.mark()
+    barrier()
+    total_ms = ev[0][0].elapsed_time(ev[-1][4])
+    per_kernel_ms = {n: sum(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps)) / args.steps
+                     for i, n in enumerate(names)}
+    sess.check_status()
+
+    # ---------------- end to end from pinned host memory
+    for _ in range(2):
+        sess.score_from_host(hb, lp_p_host, lp_s_host)
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        sess.score_from_host(hb, lp_p_host, lp_s_host)
+        torch.cuda.current_stream().synchronize()  # the caller consumes the log-probs every step
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    sess.check_status()
+    clocks = sampler.stop() if sampler else None
+
+    if world > 1:
+        tt = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(tt[0]), float(tt[1])
+        cnt = torch.tensor([wl.n_tokens, wl.n_suffix], dtype=torch.float64, device=dev)
+        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
+        job_tokens, job_suffix = float(cnt[0]), float(cnt[1])
+    else:
+        job_tokens, job_suffix = float(wl.n_tokens), float(wl.n_suffix)
+
+    if rank == 0:
+        peaks = load_peaks()
+        ms_per_step = total_ms / args.steps
+        value = job_tokens / (ms_per_step * 1e-3)
+        total_flops = sum(flops.values())
+        step_s = ms_per_step * 1e-3
+        # a step is seconds of back-to-back tensor work at the power cap: the sustained peak applies
+        peak_tf = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+        lm_ms = per_kernel_ms["lm_prefix"]
+        lm_tf = flops["lm_prefix"] / (lm_ms * 1e-3) / 1e12
+        kernels = {}
+        for n in names:
+            tf = flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12
+            kernels[n] = {"ms": round(per_kernel_ms[n], 4), "tflops": round(tf, 1),
+                          "frac_of_sustained_peak": round(tf / peak_tf, 4),
+                          "frac_of_burst_peak": round(tf / float(peaks["bf16_tflops"]), 4)}
+        line = {
+            "metric": "scored_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "prompt_tokens": wl.n_prefix,
+                       "response_tokens": wl.n_suffix, "scored_tokens_per_gpu": wl.n_tokens, "q_heads": cfg.num_q_heads,
+                       "kv_heads": cfg.num_kv_heads, "head_dim": cfg.head_dim, "hidden": cfg.hidden, "vocab": cfg.vocab,
+                       "kv_block": 16, "parallelism": f"dp{world} (independent sequences per rank, no collective)",
+                       "l2": "no flush: per-step inputs (W_vocab 1.09 GB, hidden 0.25 GB, Q/K/V 0.32 GB) exceed the 126 MB L2",
+                       "stands_in_for": cfg.stands_in_for},
+            "tflops": total_flops * world / step_s / 1e12,
+            "frac_of_bf16_peak": total_flops / step_s / 1e12 / peak_tf,
+            "response_tokens_per_s": job_suffix / step_s,
+            "kernels": kernels,
+            "roofline": {"kernel": "lm_head_partial_kernel (prompt rows; event pair spans it and its 0.1 % combine kernel)",
+                         "bound": "tensor", "achieved": lm_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": lm_tf / peak_tf,
+                         "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
+                         "frac_of_burst_peak": lm_tf / float(peaks["bf16_tflops"]),
+                         "traffic": LM_HEAD_TRAFFIC_BYTES,
+                         "algorithmic_bytes": (wl.n_prefix * cfg.hidden + cfg.vocab * cfg.hidden) * 2 + 8 * wl.n_prefix},
+            "e2e": {"value": job_tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s",
+                    "h2d_bytes_per_step": hb.nbytes(), "d2h_bytes_per_step": (wl.n_prefix + wl.n_suffix) * 4,
+                    "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": KERNELS_PER_SCORE * args.steps,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+
+            oracle.build()
+            n = args.cpu_tokens
+            t = oracle_sample(wl, n, 0)
+            line["cpu_baseline"] = {
+                "value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+                "sample": f"{n} tokens drawn uniformly from the batch ({cfg.num_q_heads} attention rows + 1 log-prob row each), {t:.1f} s"}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))
+    ap.add_argument("--cpu-tokens", type=int, default=48, help="tokens the oracle scores for cpu_baseline")
+    ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

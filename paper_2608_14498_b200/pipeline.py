@@ -1,0 +1,144 @@
+"""One scoring pass over a batch: the four library calls in the order the paper's schedule runs
+them (Section 3.1): Phase 1 = prefix attention (+ boundary-KV write) and prefix log-probs,
+Phase 2 = suffix attention over the retained KV and suffix log-probs.
+
+Only plumbing lives here (device buffers, host<->device copies, call order); all arithmetic is in
+the CUDA library.  ``ScoringSession.score`` takes tensors already on the device;
+``ScoringSession.score_from_host`` takes pinned host tensors, copies them in, runs the same calls
+and copies the log-probs back — the end-to-end path a caller with host-resident rollouts uses.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+from . import binding as B
+
+KERNELS_PER_SCORE = 6  # prefix attn, suffix attn, 2 x (LM-head partial + combine)
+
+
+@dataclass
+class Batch:
+    """Tensors of one batch (all on one device, or all pinned host tensors).
+
+    q_p/k_p/v_p: prompt tokens packed by cu_prefix; q_s/k_s/v_s: response tokens packed by
+    cu_suffix; hidden_p/ids_p and hidden_s/ids_s: final hidden rows and next-token ids scored in
+    the prefix call and in the suffix call; block_table int32 [B, max_blocks].
+    """
+
+    q_p: object
+    k_p: object
+    v_p: object
+    q_s: object
+    k_s: object
+    v_s: object
+    cu_prefix: object
+    cu_suffix: object
+    prefix_lens: object
+    block_table: object
+    hidden_p: object
+    ids_p: object
+    hidden_s: object
+    ids_s: object
+    max_prefix_len: int
+    max_suffix_len: int
+
+    def tensors(self):
+        return [self.q_p, self.k_p, self.v_p, self.q_s, self.k_s, self.v_s, self.cu_prefix, self.cu_suffix,
+                self.prefix_lens, self.block_table, self.hidden_p, self.ids_p, self.hidden_s, self.ids_s]
+
+    def nbytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in self.tensors())
+
+
+class ScoringSession:
+    """Owns the device-side state that outlives one call: W_vocab, the paged KV pool, the status
+    word, workspaces and (for host batches) staging buffers."""
+
+    def __init__(self, w_vocab, num_blocks: int, num_kv_heads: int, head_dim: int):
+        import torch
+
+        B.load_library()
+        self.torch = torch
+        self.device = w_vocab.device
+        self.w_vocab = w_vocab
+        self.k_cache = torch.zeros((num_blocks, num_kv_heads, B.BLOCK_SIZE, head_dim), dtype=torch.bfloat16,
+                                   device=self.device)
+        self.v_cache = torch.zeros_like(self.k_cache)
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self._ws = {}
+        self._staging: Optional[Batch] = None
+        self._out = {}
+
+    def _workspace(self, key: str, nbytes: int):
+        ws = self._ws.get(key)
+        if ws is None or ws.numel() < nbytes:
+            ws = self.torch.empty(max(nbytes, 16), dtype=self.torch.uint8, device=self.device)
+            self._ws[key] = ws
+        return ws
+
+    def _buf(self, key: str, shape, dtype):
+        t = self._out.get(key)
+        if t is None or tuple(t.shape) != tuple(shape) or t.dtype != dtype:
+            t = self.torch.empty(shape, dtype=dtype, device=self.device)
+            self._out[key] = t
+        return t
+
+    def score(self, b: Batch, events=None):
+        """Runs the pass on device tensors; returns (prefix log-probs, suffix log-probs, O_p, O_s).
+
+        ``events``: optional list of five CUDA events recorded before, between and after the four
+        library calls (per-kernel timing on the launching stream)."""
+        t = self.torch
+
+        def mark(i):
+            if events is not None:
+                events[i].record()
+
+        cache = (self.k_cache, self.v_cache, b.block_table)
+        code = B.RPX_BF16 if b.hidden_p.dtype == t.bfloat16 else B.RPX_F32
+        vocab, hdim = self.w_vocab.shape
+        o_p = self._buf("o_p", b.q_p.shape, b.q_p.dtype)
+        o_s = self._buf("o_s", b.q_s.shape, b.q_s.dtype)
+        lp_p = self._buf("lp_p", (b.hidden_p.shape[0],), t.float32)
+        lp_s = self._buf("lp_s", (b.hidden_s.shape[0],), t.float32)
+        mark(0)
+        B.prefix_attn(b.q_p, b.k_p, b.v_p, b.cu_prefix, b.max_prefix_len, cache=cache, out=o_p,
+                      workspace=self._workspace("attn", B.prefix_attn_workspace_bytes(
+                          b.q_p.shape[1], b.k_p.shape[1], b.q_p.shape[2], B._dtype_code(b.q_p), b.q_p.shape[0])),
+                      device_status=self.status)
+        mark(1)
+        B.token_logprobs(b.hidden_p, self.w_vocab, b.ids_p, logprobs=lp_p, device_status=self.status,
+                         workspace=self._workspace("lm", B.token_logprobs_workspace_bytes(
+                             b.hidden_p.shape[0], hdim, vocab, code)))
+        mark(2)
+        B.suffix_attn(b.q_s, b.k_s, b.v_s, b.cu_suffix, b.prefix_lens, b.max_suffix_len, b.max_prefix_len, cache=cache,
+                      out=o_s, workspace=self._workspace("attn", B.suffix_attn_workspace_bytes(
+                          b.q_s.shape[1], b.k_s.shape[1], b.q_s.shape[2], B._dtype_code(b.q_s), b.q_s.shape[0])),
+                      device_status=self.status)
+        mark(3)
+        B.token_logprobs(b.hidden_s, self.w_vocab, b.ids_s, logprobs=lp_s, device_status=self.status,
+                         workspace=self._workspace("lm", B.token_logprobs_workspace_bytes(
+                             b.hidden_s.shape[0], hdim, vocab, code)))
+        mark(4)
+        return lp_p, lp_s, o_p, o_s
+
+    def score_from_host(self, hb: Batch, lp_p_host, lp_s_host):
+        """Pinned host batch in, log-probs out into the pinned ``lp_*_host`` tensors.  Copies and
+        kernels are enqueued on the current stream; the caller synchronises."""
+        t = self.torch
+        if self._staging is None or any(tuple(a.shape) != tuple(c.shape) or a.dtype != c.dtype
+                                        for a, c in zip(self._staging.tensors(), hb.tensors())):
+            dev = [t.empty(x.shape, dtype=x.dtype, device=self.device) for x in hb.tensors()]
+            self._staging = Batch(*dev, hb.max_prefix_len, hb.max_suffix_len)
+        for dst, src in zip(self._staging.tensors(), hb.tensors()):
+            dst.copy_(src, non_blocking=True)
+        lp_p, lp_s, _, _ = self.score(self._staging)
+        lp_p_host.copy_(lp_p, non_blocking=True)
+        lp_s_host.copy_(lp_s, non_blocking=True)
+        return lp_p_host, lp_s_host
+
+    def check_status(self) -> None:
+        code = int(self.status.item())
+        if code != 0:
+            raise B.RpxError(code, "device status")
