@@ -144,6 +144,35 @@ RPX_API rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_s
                                 void* workspace, size_t workspace_bytes, int32_t* device_status,
                                 void* cuda_stream);
 
+/*
+ * Allocation-free variant of rpx_token_logprobs (the paper has no counterpart: this entry point
+ * exists for deployment, not for the method).  It is meant for callers that cannot give the
+ * library a workspace because they cannot allocate one: a scoring hook that runs inside an
+ * engine which has already handed every free byte of HBM to its KV pool (the co-located
+ * rollout/training setting), or a section of a serving loop where calling the device allocator is
+ * off limits because cudaMalloc may fail there or stall the whole device while it runs.
+ *
+ * The per-(vocab chunk, row) partial records that rpx_token_logprobs keeps in the caller's
+ * workspace live here in a fixed array of RPX_STATIC_SCRATCH_BYTES inside the library image;
+ * every GPU that loads the library holds that array until the process exits.  Inputs and outputs
+ * are still the caller's.  bf16 inputs only; same result as rpx_token_logprobs.
+ *   - Limit: ceil(ceil(vocab / 256) / 16) * n_tokens * 16 bytes must not exceed
+ *     RPX_STATIC_SCRATCH_BYTES (vocab 152064 => at most 13797 rows per call); larger problems
+ *     return RPX_ERR_WORKSPACE before any launch — split the rows over several calls.
+ *   - The first call on each device looks up the array's device address (one host-side runtime
+ *     query, no allocation).  Make that first call before starting any stream capture.
+ *   - Every call on a device shares the one array, which keeps the previous call's contents.
+ *     Nothing in it has to start at zero (each call overwrites every record it later reads), but
+ *     two calls that overlap on the GPU (different streams, or different threads) race on it:
+ *     issue them on one stream or serialise them yourself.
+ *   - No cudaMalloc, cudaFree or allocating library routine is called.
+ */
+#define RPX_STATIC_SCRATCH_BYTES (8u << 20)
+RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                               const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
+                                               int32_t vocab, float* logprobs, float* lse, int32_t* device_status,
+                                               void* cuda_stream);
+
 /* Workspace sizes in bytes for the calls above (pure host arithmetic; 0 is possible). */
 RPX_API size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens);
 RPX_API size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens);

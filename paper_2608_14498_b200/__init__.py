@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     suffix_attn,
     suffix_attn_workspace_bytes,
     token_logprobs,
+    token_logprobs_static,
     token_logprobs_workspace_bytes,
     version,
 )

@@ -16,11 +16,13 @@ _lib = None
 
 RPX_BF16, RPX_F32 = 0, 1
 BLOCK_SIZE = 16
+STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = (
     "rpx_prefix_attn",
     "rpx_suffix_attn",
     "rpx_token_logprobs",
+    "rpx_token_logprobs_static",
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
     "rpx_token_logprobs_workspace_bytes",
@@ -80,6 +82,8 @@ def load_library():
                                     i32, ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs.restype = i32
     lib.rpx_token_logprobs.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_static.restype = i32
+    lib.rpx_token_logprobs_static.argtypes = [vp, i64, vp, vp, i64, i32, i32, vp, vp, vp, vp]
     lib.rpx_prefix_attn_workspace_bytes.restype = sz
     lib.rpx_prefix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
     lib.rpx_suffix_attn_workspace_bytes.restype = sz
@@ -252,3 +256,28 @@ def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_
     if rc != 0:
         raise RpxError(rc, "rpx_token_logprobs")
     return (logprobs, lse) if return_lse else logprobs
+
+
+def token_logprobs_static(hidden, w_vocab, target_ids, logprobs, lse=None, device_status=None, stream=None):
+    """rpx_token_logprobs_static: the same log-probs, for callers that cannot allocate device memory.
+
+    Nothing is allocated on this path, not even by torch: ``logprobs`` (float32 [N]) must be passed
+    in, and the partial records go to a fixed array inside the library.  Use it where the device
+    allocator is out of reach (all HBM already reserved by the host engine, or a code section in
+    which an allocator call could fail or stall the device).  bf16 only; the problem must fit
+    ``STATIC_SCRATCH_BYTES`` (raises RpxError RPX_ERR_WORKSPACE otherwise); calls that overlap on
+    the GPU race on the shared array.
+    """
+    lib = load_library()
+    if _dtype_code(hidden) != RPX_BF16 or _dtype_code(w_vocab) != RPX_BF16:
+        raise TypeError("the allocation-free entry point takes bfloat16 tensors only")
+    if hidden.dim() != 2 or hidden.stride(1) != 1 or not w_vocab.is_contiguous():
+        raise ValueError("hidden must be [N, H] with contiguous rows and w_vocab contiguous [V, H]")
+    n, hdim = hidden.shape
+    row_stride = hidden.stride(0) if n > 1 else hdim
+    rc = lib.rpx_token_logprobs_static(_ptr(hidden), row_stride, _ptr(w_vocab), _ptr(target_ids), n, hdim,
+                                       w_vocab.shape[0], _ptr(logprobs), _ptr(lse), _ptr(device_status),
+                                       _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_token_logprobs_static")
+    return logprobs

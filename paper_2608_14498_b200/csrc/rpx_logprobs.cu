@@ -15,6 +15,8 @@
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "rpx_internal.h"
 #include "rpx_ptx.cuh"
 
@@ -341,3 +343,72 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
 }
 
 }  // namespace rpx
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant.  The partial (max, sum, target-logit) records normally live in the
+// caller's workspace; here they live in a fixed array inside the library image, so a caller that
+// has no device memory left to hand over (or must not touch the allocator) can still score.
+// ---------------------------------------------------------------------------------------------
+namespace rpx {
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[RPX_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the CURRENT device.  In host code the array's name is only
+// a handle for the runtime, not a device address; the address has to be asked for, per device.
+rpx_status_t static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RPX_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return RPX_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return RPX_OK;
+}
+
+}  // namespace
+}  // namespace rpx
+
+extern "C" RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, int64_t hidden_row_stride,
+                                                          const void* w_vocab, const int32_t* target_ids,
+                                                          int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                                          float* logprobs, float* lse, int32_t* device_status,
+                                                          void* cuda_stream) {
+    using namespace rpx;
+    if (n_tokens < 0 || n_tokens >= INT32_MAX || hidden_dim <= 0 || vocab <= 0 || hidden_dim % 8 != 0)
+        return RPX_ERR_SHAPE;
+    if (n_tokens == 0) return RPX_OK;
+    if (hidden == nullptr || w_vocab == nullptr || target_ids == nullptr || logprobs == nullptr) return RPX_ERR_NULL;
+    if (hidden_row_stride < hidden_dim) return RPX_ERR_SHAPE;
+    if (hidden_row_stride % 8 != 0) return RPX_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0 || (reinterpret_cast<uintptr_t>(w_vocab) & 15u) != 0)
+        return RPX_ERR_ALIGN;
+    // one 16-byte record per (vocab chunk, row) must fit in the built-in array
+    const size_t need = static_cast<size_t>(logprob_num_chunks(vocab)) * static_cast<size_t>(n_tokens) * sizeof(float4);
+    if (need > static_cast<size_t>(RPX_STATIC_SCRATCH_BYTES)) return RPX_ERR_WORKSPACE;
+    if (rpx_status_t rc = check_arch()) return rc;
+    void* scratch = nullptr;
+    if (rpx_status_t rc = static_scratch_for_current_device(&scratch)) return rc;
+
+    LogprobArgs a;
+    a.hidden = hidden;
+    a.hidden_row_stride = hidden_row_stride;
+    a.w = w_vocab;
+    a.target_ids = target_ids;
+    a.n_tokens = n_tokens;
+    a.hidden_dim = hidden_dim;
+    a.vocab = vocab;
+    a.logprobs = logprobs;
+    a.lse = lse;
+    a.partials = scratch;
+    a.device_status = device_status;
+    a.stream = static_cast<cudaStream_t>(cuda_stream);
+    return launch_token_logprobs(a);
+}
