@@ -6,13 +6,17 @@
 // unmasked except the last partial one), then the self tiles up to each query tile's diagonal.
 //   warps 0-3 : softmax of query tile 0   (thread = one row; TMEM lane = row)
 //   warps 4-7 : softmax of query tile 1
-//   warp  8   : TMA producer (Q once; K/V through a 3-slot ring; paged tiles = one TMA box per
+//   warp  8   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
 //               16-token page); it also stores the diagonal K/V tiles into the paged cache
 //   warp  9   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
-//               O_t += P_t V (P_t bf16 in swizzled smem, V as an MN-major operand)
-// The two query tiles alternate on the tensor core: while the softmax warps of one tile work on
-// S_t(j), the tensor core runs the other tile's PV(j-1) and QK(j).  Scores are kept in log2
-// units; O is rescaled lazily (only when a row's running max grows by more than 2^8).
+//               O_t += P_t V  (P_t = bf16 probabilities written back into the first 64 columns
+//               of S_t's TMEM region and consumed as the TMEM A operand; V straight from its
+//               [keys][d] tile as an MN-major B operand)
+// The two query tiles alternate on the tensor core in the order PV_0(j) QK_0(j+1) PV_1(j)
+// QK_1(j+1): while the softmax warps of one tile work on S_t, the tensor core runs the other
+// tile's two MMAs; issuing PV_t(j) before QK_t(j+1) also orders the read of P_t before the
+// overwrite of S_t.  Scores are kept in log2 units; O is rescaled lazily (only when a row's
+// running max grows by more than 2^8).
 #include <math_constants.h>
 
 #include "rpx_internal.h"
@@ -23,7 +27,7 @@ namespace rpx {
 namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
-constexpr int kSlots = 3;
+constexpr int kSlots = 5;
 constexpr int kThreads = 320;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -34,9 +38,9 @@ struct Ctl {
     uint64_t q_full;
     uint64_t kv_full[kSlots];
     uint64_t kv_empty[kSlots];
-    uint64_t s_full[2];
-    uint64_t p_ready[2];
-    uint64_t pv_done[2];
+    uint64_t s_full[2];   // tensor core -> softmax: S_t(j) is in TMEM (and PV_t(j-1) has finished)
+    uint64_t p_ready[2];  // softmax -> tensor core: P_t(j) is in TMEM, O_t rescaled if needed
+    uint64_t o_done[2];   // tensor core -> softmax: the last PV_t has finished
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -50,10 +54,8 @@ struct Layout {
     static constexpr int kHalfBytes = kTileK * 128;      // one [128 rows][64 bf16] swizzled block
     static constexpr int kQBytes = kHalves * kHalfBytes; // one query tile
     static constexpr int kKvBytes = kHalves * kHalfBytes;
-    static constexpr int kPBytes = 2 * kHalfBytes;       // [128 rows][128 keys] bf16
     static constexpr int kQOff = 0;
-    static constexpr int kPOff = 2 * kQBytes;
-    static constexpr int kKvOff = kPOff + 2 * kPBytes;
+    static constexpr int kKvOff = 2 * kQBytes;
     static constexpr int kCtlOff = kKvOff + kSlots * kKvBytes;
     static constexpr size_t kSmemBytes = 1024 + kCtlOff + sizeof(Ctl);
 };
@@ -120,7 +122,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         for (int t = 0; t < 2; ++t) {
             mbar_init(&ctl->s_full[t], 1);
             mbar_init(&ctl->p_ready[t], 128);
-            mbar_init(&ctl->pv_done[t], 1);
+            mbar_init(&ctl->o_done[t], 1);
         }
         mbar_init(&ctl->drain, 1);
         ctl->abort_flag = 0;
@@ -277,7 +279,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             constexpr uint32_t idesc_qk = make_idesc_bf16(kTileQ, kTileK, false, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(kTileQ, D, false, true);
             const uint32_t q_addr = smem_u32(smem + L::kQOff);
-            const uint32_t p_addr = smem_u32(smem + L::kPOff);
             const uint32_t kv_addr = smem_u32(smem + L::kKvOff);
             bool ok = true;
 
@@ -292,15 +293,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 umma_commit(&ctl->s_full[t]);
             };
             auto issue_pv = [&](int t, uint32_t v_slot, bool accumulate) {
-                const uint32_t a0 = p_addr + t * L::kPBytes, b0 = kv_addr + v_slot * L::kKvBytes;
+                const uint32_t b0 = kv_addr + v_slot * L::kKvBytes;
 #pragma unroll
                 for (int k = 0; k < kTileK / 16; ++k) {
-                    const uint32_t a_off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
-                    umma_bf16_ss(tmem_o[t], make_smem_desc_sw128(a0 + a_off, 16, 1024),
-                                 make_smem_desc_sw128(b0 + k * 2048, L::kHalfBytes, 1024), idesc_pv,
-                                 (accumulate || k != 0) ? 1u : 0u);
+                    // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
+                    umma_bf16_ts(tmem_o[t], tmem_s[t] + k * 8, make_smem_desc_sw128(b0 + k * 2048, L::kHalfBytes, 1024),
+                                 idesc_pv, (accumulate || k != 0) ? 1u : 0u);
                 }
-                umma_commit(&ctl->pv_done[t]);
             };
 
             ok = mbar_wait(&ctl->q_full, 0, abort_flag);
@@ -321,7 +320,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         ok = false;
                         break;
                     }
+                    if (!have_v) {
+                        if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        have_v = true;
+                    }
                     tc_fence_after_sync();
+                    issue_pv(t, v_slot, j != 0);
                     if (j + 1 < n_tile[t]) {
                         if (!have_kn) {
                             if (!mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag)) {
@@ -331,21 +338,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                             tc_fence_after_sync();
                             have_kn = true;
                         }
-                        issue_qk(t, kn_slot);
+                        issue_qk(t, kn_slot);  // in order behind PV_t(j): P_t is read before S_t is rewritten
+                    } else {
+                        umma_commit(&ctl->o_done[t]);
                     }
-                    if (!have_v) {
-                        if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after_sync();
-                        have_v = true;
-                    }
-                    issue_pv(t, v_slot, j != 0);
                 }
                 if (!ok) break;
-                if (have_kn) umma_commit(&ctl->kv_empty[kn_slot]);
                 umma_commit(&ctl->kv_empty[v_slot]);
+                if (have_kn) umma_commit(&ctl->kv_empty[kn_slot]);
             }
             if (!ok) {
                 umma_commit(&ctl->drain);
@@ -361,7 +361,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             const int32_t row = quarter * 32 + lane;
             const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
             const uint32_t lane_addr = (quarter * 32u) << 16;
-            uint8_t* p_smem = smem + L::kPOff + t * L::kPBytes;
             float run_max = -CUDART_INF_F, run_sum = 0.f;
             bool ok = true;
             for (int32_t j = 0; j < n_tile[t]; ++j) {
@@ -370,6 +369,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     break;
                 }
                 tc_fence_after_sync();
+                // ---- the row's 128 scores
+                uint32_t sc[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s[t] + c * 32 + lane_addr, sc[c]);
+                tmem_ld_wait();
                 // ---- how many leading keys of this tile the row may see
                 int32_t n_vis;
                 if (j < n_prefix_tiles) {
@@ -378,74 +382,58 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     const int32_t jt = j - n_prefix_tiles;
                     n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
                 }
-                // ---- pass 1: row maximum (log2 units)
-                float cmax = -CUDART_INF_F;
-#pragma unroll 1
-                for (int c = 0; c < kTileK / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_s[t] + c * 32 + lane_addr, r);
-                    tmem_ld_wait();
+                if (n_vis < kTileK) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float x = __uint_as_float(r[i]);
-                        cmax = fmaxf(cmax, (c * 32 + i < n_vis) ? x : -CUDART_INF_F);
-                    }
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (c * 32 + i >= n_vis) sc[c][i] = 0xff800000u;  // -inf
                 }
+                float cmax = -CUDART_INF_F;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) cmax = fmaxf(cmax, __uint_as_float(sc[c][i]));
                 cmax *= p.scale_log2;  // scale > 0, so max commutes with the scaling
                 const bool grow = cmax > run_max + kRescaleThreshold;
                 const float new_max = grow ? cmax : run_max;
-                if (j > 0) {
-                    if (!mbar_wait(&ctl->pv_done[t], (j - 1) & 1, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after_sync();
-                    if (__any_sync(0xffffffffu, grow)) {
-                        const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
+                // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent here
+                if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                    const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
 #pragma unroll 1
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
-                            tmem_ld_wait();
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
+                        tmem_ld_wait();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                            tmem_st32(tmem_o[t] + c * 32 + lane_addr, r);
-                        }
-                        tmem_st_wait();
-                        run_sum *= alpha;
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(tmem_o[t] + c * 32 + lane_addr, r);
                     }
+                    run_sum *= alpha;
                 }
                 run_max = new_max;
-                // ---- pass 2: P = 2^(x - max) as bf16 into swizzled smem, row sum in fp32
+                // ---- P = 2^(x - max) as packed bf16 pairs over the first 64 columns of S_t
                 const float neg_max = -run_max;
                 float part = 0.f;
-#pragma unroll 1
-                for (int c = 0; c < kTileK / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_s[t] + c * 32 + lane_addr, r);
-                    tmem_ld_wait();
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        float e0 = fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_max));
-                        float e1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_max));
-                        e0 = (c * 32 + i < n_vis) ? e0 : 0.f;
-                        e1 = (c * 32 + i + 1 < n_vis) ? e1 : 0.f;
+                        const float e0 = fast_exp2(fmaf(__uint_as_float(sc[c][i]), p.scale_log2, neg_max));
+                        const float e1 = fast_exp2(fmaf(__uint_as_float(sc[c][i + 1]), p.scale_log2, neg_max));
                         part += e0 + e1;
                         packed[i >> 1] = pack_bf16x2(e0, e1);
                     }
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        *reinterpret_cast<uint4*>(p_smem + swz_off(row, c * 4 + q4)) =
-                            make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
+                    tmem_st16(tmem_s[t] + c * 16 + lane_addr, packed);
                 }
                 run_sum += part;
-                fence_proxy_async_smem();
+                tmem_st_wait();
                 tc_fence_before_sync();
                 mbar_arrive(&ctl->p_ready[t]);
             }
             // ---- epilogue: O / l -> global, LSE
-            if (ok && mbar_wait(&ctl->pv_done[t], (n_tile[t] - 1) & 1, abort_flag)) {
+            if (ok && mbar_wait(&ctl->o_done[t], 0, abort_flag)) {
                 tc_fence_after_sync();
                 const bool row_valid = q_local < len_q;
                 const float inv = 1.f / run_sum;
