@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return _OUT
     tmp = _OUT + f".tmp{os.getpid()}"
     cmd = [
-        _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--shared",
+        _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "--use_fast_math", "-std=c++17", "--shared",
         "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-cudart", "static",
         "-I", os.path.join(_ROOT, "include"), "-I", _CSRC,
     ]

@@ -4,11 +4,14 @@
 // One CTA owns two adjacent 128-row query tiles of one (sequence, query head) and walks the key
 // tiles (128 keys) that those rows may see: first the cached prefix tiles (suffix pass only,
 // unmasked except the last partial one), then the self tiles up to each query tile's diagonal.
-//   warps 0-3 : softmax of query tile 0   (thread = one row; TMEM lane = row)
-//   warps 4-7 : softmax of query tile 1
-//   warp  8   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
+//   warps 0-7  : softmax of query tile 0: warp w owns rows 32*(w%4).. (its TMEM lane quarter) and
+//                key columns 64*(w/4)..+63, so two threads share a row and twice as many warps
+//                hide each other's latencies; the pair exchanges its row maximum (and, at the
+//                end, its row sum) through shared memory and a 64-thread mbarrier
+//   warps 8-15 : softmax of query tile 1
+//   warp  16   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
 //               16-token page); it also stores the diagonal K/V tiles into the paged cache
-//   warp  9   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
+//   warp  17   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
 //               O_t += P_t V  (P_t = bf16 probabilities written back into the first 64 columns
 //               of S_t's TMEM region and consumed as the TMEM A operand; V straight from its
 //               [keys][d] tile as an MN-major B operand)
@@ -28,7 +31,8 @@ namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
 constexpr int kSlots = 5;
-constexpr int kThreads = 320;
+constexpr int kThreads = 576;
+constexpr int kProducerWarp = 16, kMmaWarp = 17;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -41,11 +45,13 @@ struct Ctl {
     uint64_t s_full[2];   // tensor core -> softmax: S_t(j) is in TMEM (and PV_t(j-1) has finished)
     uint64_t p_ready[2];  // softmax -> tensor core: P_t(j) is in TMEM, O_t rescaled if needed
     uint64_t o_done[2];   // tensor core -> softmax: the last PV_t has finished
+    uint64_t pair_sync[2][4];  // the two warps sharing rows 32q..32q+31 of tile t
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t drain_flag;
     uint32_t data_error;
+    float xchg[2][2][128];     // [tile][column half][row]: row maximum, later row sum
 };
 
 template <int D>
@@ -57,7 +63,7 @@ struct Layout {
     static constexpr int kQOff = 0;
     static constexpr int kKvOff = 2 * kQBytes;
     static constexpr int kCtlOff = kKvOff + kSlots * kKvBytes;
-    static constexpr size_t kSmemBytes = 1024 + kCtlOff + sizeof(Ctl);
+    static constexpr size_t kSmemBytes = kCtlOff + sizeof(Ctl);  // the dynamic window is declared 1024-aligned
 };
 
 struct Params {
@@ -103,11 +109,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     const int32_t len_p = p.prefix_lens != nullptr ? p.prefix_lens[seq] : 0;
     const bool active1 = q0 + kTileQ < len_q;
     const int32_t n_prefix_tiles = (len_p + kTileK - 1) / kTileK;
-    const int32_t n_tile[2] = {n_prefix_tiles + 2 * pair + 1, n_prefix_tiles + 2 * pair + 2};
-    const int32_t n_kv = active1 ? n_tile[1] : n_tile[0];
+    // key tiles seen by query tile t: n_tile0 + t.  (Scalars, not arrays: a small array indexed at
+    // run time lives in local memory, and with nearly all L1 carved out as shared memory every such
+    // load stalls the in-order warp for hundreds of cycles.)
+    const int32_t n_tile0 = n_prefix_tiles + 2 * pair + 1;
+    const int32_t n_kv = active1 ? n_tile0 + 1 : n_tile0;
 
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if ((smem_u32(smem) & 1023u) != 0u) {  // swizzled tiles need 1024-byte alignment; never expected
+        if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, RPX_ERR_CUDA);
+        return;
+    }
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + L::kCtlOff);
     volatile uint32_t* abort_flag = &ctl->abort_flag;
     const int warp = threadIdx.x >> 5;
@@ -121,8 +133,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&ctl->s_full[t], 1);
-            mbar_init(&ctl->p_ready[t], 128);
+            mbar_init(&ctl->p_ready[t], 8);  // one arrival per softmax warp
             mbar_init(&ctl->o_done[t], 1);
+            for (int q = 0; q < 4; ++q) mbar_init(&ctl->pair_sync[t][q], 2);  // one arrival per warp of the pair
         }
         mbar_init(&ctl->drain, 1);
         ctl->abort_flag = 0;
@@ -130,7 +143,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         ctl->data_error = 0;
         fence_barrier_init();
     }
-    if (warp == 9) {
+    if (warp == kMmaWarp) {
         tmem_alloc(&ctl->tmem_base, kTmemCols);
         tmem_relinquish();
     }
@@ -138,10 +151,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
-    const uint32_t tmem_s[2] = {tmem_base, tmem_base + 128};
-    const uint32_t tmem_o[2] = {tmem_base + 256, tmem_base + 384};
+    // TMEM columns: S_t at 128 t (P_t aliases its first 64), O_t at 256 + 128 t
 
-    if (warp == 8) {
+    if (warp == kProducerWarp) {
         // =========================================================== producer warp
         bool ok = true;
         if (lane == 0) {
@@ -159,10 +171,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         for (int32_t j = 0; ok && j < n_kv; ++j) {
             const bool from_cache = j < n_prefix_tiles;
             const int32_t jt = from_cache ? j : j - n_prefix_tiles;  // tile index inside its key source
-            uint32_t slot_of[2];
+            uint32_t slot_k = 0, slot_v = 0;
             for (int which = 0; which < 2; ++which, ++n_loaded) {  // 0 = K, 1 = V
                 const uint32_t slot = n_loaded % kSlots, phase = (n_loaded / kSlots) & 1u;
-                slot_of[which] = slot;
+                if (which == 0) slot_k = slot; else slot_v = slot;
                 if (!mbar_wait(&ctl->kv_empty[slot], phase ^ 1u, abort_flag)) {
                     ok = false;
                     break;
@@ -222,7 +234,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (ok && owns_cache_write && !from_cache && jt >= 2 * pair) {
                 for (int which = 0; which < 2 && ok; ++which) {
                     const uint32_t idx = n_loaded - 2 + which;
-                    const uint32_t slot = slot_of[which];
+                    const uint32_t slot = which == 0 ? slot_k : slot_v;
                     if (!mbar_wait(&ctl->kv_full[slot], (idx / kSlots) & 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -270,10 +282,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             // abort: give copies already in flight a moment to land before smem is released
             const uint32_t first = n_loaded > kSlots ? n_loaded - kSlots : 0u;
             for (uint32_t i = first; i < n_loaded; ++i)
-                mbar_wait(&ctl->kv_full[i % kSlots], (i / kSlots) & 1u, &ctl->drain_flag, 1000000ull);
-            mbar_wait(&ctl->q_full, 0, &ctl->drain_flag, 1000000ull);
+                mbar_wait(&ctl->kv_full[i % kSlots], (i / kSlots) & 1u, &ctl->drain_flag, kDrainLimitCycles);
+            mbar_wait(&ctl->q_full, 0, &ctl->drain_flag, kDrainLimitCycles);
         }
-    } else if (warp == 9) {
+    } else if (warp == kMmaWarp) {
         // =========================================================== tcgen05 issuer (one thread)
         if (elect_one()) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(kTileQ, kTileK, false, false);
@@ -282,24 +294,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             const uint32_t kv_addr = smem_u32(smem + L::kKvOff);
             bool ok = true;
 
+            // descriptors: everything but the start address is constant, so keep bases and add offsets
+            const uint64_t q_desc0 = make_smem_desc_sw128(q_addr, 16, 1024);
+            const uint64_t k_desc0 = make_smem_desc_sw128(kv_addr, 16, 1024);             // K tile: K-major
+            const uint64_t v_desc0 = make_smem_desc_sw128(kv_addr, L::kHalfBytes, 1024);  // V tile: MN-major
             auto issue_qk = [&](int t, uint32_t k_slot) {
-                const uint32_t a0 = q_addr + t * L::kQBytes, b0 = kv_addr + k_slot * L::kKvBytes;
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k >> 2) * L::kHalfBytes + (k & 3) * 32;
-                    umma_bf16_ss(tmem_s[t], make_smem_desc_sw128(a0 + off, 16, 1024),
-                                 make_smem_desc_sw128(b0 + off, 16, 1024), idesc_qk, k != 0 ? 1u : 0u);
-                }
+                const uint64_t kd = k_desc0 + static_cast<uint64_t>(k_slot * (L::kKvBytes >> 4));
+                const uint64_t qd = q_desc0 + static_cast<uint64_t>(t * (L::kQBytes >> 4));
+                if (D == 128) umma_ss_k128_overwrite(tmem_base + t * 128, qd, kd, idesc_qk);
+                else umma_ss_k64_overwrite(tmem_base + t * 128, qd, kd, idesc_qk);
                 umma_commit(&ctl->s_full[t]);
             };
             auto issue_pv = [&](int t, uint32_t v_slot, bool accumulate) {
-                const uint32_t b0 = kv_addr + v_slot * L::kKvBytes;
-#pragma unroll
-                for (int k = 0; k < kTileK / 16; ++k) {
-                    // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
-                    umma_bf16_ts(tmem_o[t], tmem_s[t] + k * 8, make_smem_desc_sw128(b0 + k * 2048, L::kHalfBytes, 1024),
-                                 idesc_pv, (accumulate || k != 0) ? 1u : 0u);
-                }
+                // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
+                umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128,
+                             v_desc0 + static_cast<uint64_t>(v_slot * (L::kKvBytes >> 4)), idesc_pv,
+                             accumulate ? 1u : 0u);
             };
 
             ok = mbar_wait(&ctl->q_full, 0, abort_flag);
@@ -315,7 +325,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const uint32_t v_slot = v_idx % kSlots, kn_slot = kn_idx % kSlots;
                 bool have_v = false, have_kn = false;
                 for (int t = 0; t < 2 && ok; ++t) {
-                    if ((t == 1 && !active1) || j >= n_tile[t]) continue;
+                    if ((t == 1 && !active1) || j >= n_tile0 + t) continue;
                     if (!mbar_wait(&ctl->p_ready[t], j & 1, abort_flag)) {
                         ok = false;
                         break;
@@ -329,7 +339,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     }
                     tc_fence_after_sync();
                     issue_pv(t, v_slot, j != 0);
-                    if (j + 1 < n_tile[t]) {
+                    if (j + 1 < n_tile0 + t) {
                         if (!have_kn) {
                             if (!mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag)) {
                                 ok = false;
@@ -349,32 +359,39 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             }
             if (!ok) {
                 umma_commit(&ctl->drain);
-                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, 1000000ull);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, kDrainLimitCycles);
             }
         }
         __syncwarp();
     } else {
         // =========================================================== softmax warps
-        const int t = warp >> 2;
+        const int t = warp >> 3;
         if (t == 0 || active1) {
             const uint32_t quarter = warp & 3;
+            const int half = (warp >> 2) & 1;
             const int32_t row = quarter * 32 + lane;
             const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
             const uint32_t lane_addr = (quarter * 32u) << 16;
+            uint64_t* pair_bar = &ctl->pair_sync[t][quarter];
+            float* my_slot = &ctl->xchg[t][half][row];
+            const float* peer_slot = &ctl->xchg[t][half ^ 1][row];
+            const int32_t my_tiles = n_tile0 + t;
+            const uint32_t my_s = tmem_base + t * 128 + lane_addr;        // this thread's lane of S_t / P_t
+            const uint32_t my_o = tmem_base + 256 + t * 128 + lane_addr;  // and of O_t
             float run_max = -CUDART_INF_F, run_sum = 0.f;
             bool ok = true;
-            for (int32_t j = 0; j < n_tile[t]; ++j) {
+            for (int32_t j = 0; j < my_tiles; ++j) {
                 if (!mbar_wait(&ctl->s_full[t], j & 1, abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after_sync();
-                // ---- the row's 128 scores
-                uint32_t sc[4][32];
+                // ---- this thread's 64 scores of the row
+                uint32_t sc[2][32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s[t] + c * 32 + lane_addr, sc[c]);
+                for (int c = 0; c < 2; ++c) tmem_ld32(my_s + half * 64 + c * 32, sc[c]);
                 tmem_ld_wait();
-                // ---- how many leading keys of this tile the row may see
+                // ---- how many leading keys of this tile the row may see, counted from this half
                 int32_t n_vis;
                 if (j < n_prefix_tiles) {
                     n_vis = min(kTileK, len_p - j * kTileK);
@@ -382,66 +399,100 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     const int32_t jt = j - n_prefix_tiles;
                     n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
                 }
-                if (n_vis < kTileK) {
+                n_vis -= half * 64;
+                if (n_vis < 64) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < 2; ++c)
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (c * 32 + i >= n_vis) sc[c][i] = 0xff800000u;  // -inf
                 }
-                float cmax = -CUDART_INF_F;
+                // eight independent chains: a row maximum is latency-bound, not throughput-bound
+                float mx[8];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int u = 0; u < 8; ++u) mx[u] = -CUDART_INF_F;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) cmax = fmaxf(cmax, __uint_as_float(sc[c][i]));
-                cmax *= p.scale_log2;  // scale > 0, so max commutes with the scaling
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8)
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(sc[c][i + u]));
+                float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                   fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                // ---- agree on the row maximum with the thread that holds the other 64 columns.  The
+                // barrier also orders both threads' S loads before either thread's P stores, which
+                // land on columns the other thread reads its scores from.
+                *my_slot = cmax;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pair_bar);  // a warp-wide arrival: 256 single arrivals per step
+                                                       // would serialise on the barrier word
+                if (!mbar_wait(pair_bar, j & 1, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                cmax = fmaxf(cmax, *peer_slot) * p.scale_log2;  // scale > 0, so max commutes with the scaling
                 const bool grow = cmax > run_max + kRescaleThreshold;
                 const float new_max = grow ? cmax : run_max;
-                // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent here
-                if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                    const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
-#pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st32(tmem_o[t] + c * 32 + lane_addr, r);
-                    }
-                    run_sum *= alpha;
-                }
+                const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
+                const bool rescale = j > 0 && __any_sync(0xffffffffu, grow);
+                run_sum *= alpha;
                 run_max = new_max;
                 // ---- P = 2^(x - max) as packed bf16 pairs over the first 64 columns of S_t
                 const float neg_max = -run_max;
-                float part = 0.f;
+                float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
                         const float e0 = fast_exp2(fmaf(__uint_as_float(sc[c][i]), p.scale_log2, neg_max));
                         const float e1 = fast_exp2(fmaf(__uint_as_float(sc[c][i + 1]), p.scale_log2, neg_max));
-                        part += e0 + e1;
+                        part[(i / 2) % 4] += e0 + e1;
                         packed[i >> 1] = pack_bf16x2(e0, e1);
                     }
-                    tmem_st16(tmem_s[t] + c * 16 + lane_addr, packed);
+                    tmem_st16(my_s + half * 32 + c * 16, packed);
                 }
-                run_sum += part;
+                run_sum += (part[0] + part[1]) + (part[2] + part[3]);
+                // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent until this warp's arrival
+                // below; each thread of the pair rescales its half of the row's O columns.  Done here,
+                // after the scores are dead, so the 32 staging registers do not force spills.
+                if (rescale) {
+#pragma unroll 1
+                    for (int c = 0; c < D / 64; ++c) {
+                        uint32_t r[32];
+                        const uint32_t addr = my_o + half * (D / 2) + c * 32;
+                        tmem_ld32(addr, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(addr, r);
+                    }
+                }
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(&ctl->p_ready[t]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->p_ready[t]);
             }
-            // ---- epilogue: O / l -> global, LSE
-            if (ok && mbar_wait(&ctl->o_done[t], 0, abort_flag)) {
+            // ---- epilogue: O / l -> global, LSE; each thread of the pair writes half of the row
+            if (ok) ok = mbar_wait(&ctl->o_done[t], 0, abort_flag);
+            if (ok) {
+                // the last PV ran after every thread's last p_ready arrival, hence after the partner
+                // read this thread's last maximum: the slot can now carry the row sum
+                *my_slot = run_sum;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pair_bar);
+                ok = mbar_wait(pair_bar, my_tiles & 1, abort_flag);
+            }
+            if (ok) {
                 tc_fence_after_sync();
+                run_sum += *peer_slot;
                 const bool row_valid = q_local < len_q;
                 const float inv = 1.f / run_sum;
-                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
+                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D + half * (D / 2);
 #pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
+                for (int c = 0; c < D / 64; ++c) {
                     uint32_t r[32];
-                    tmem_ld32(tmem_o[t] + c * 32 + lane_addr, r);
+                    tmem_ld32(my_o + half * (D / 2) + c * 32, r);
                     tmem_ld_wait();
                     if (row_valid) {
                         if (p.out_f32) {
@@ -464,7 +515,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         }
                     }
                 }
-                if (row_valid && p.lse != nullptr)
+                if (half == 0 && row_valid && p.lse != nullptr)
                     p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
             }
         }
@@ -472,7 +523,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }

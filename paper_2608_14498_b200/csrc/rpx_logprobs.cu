@@ -139,7 +139,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                 // abort: let the copies already in flight land before the CTA's smem goes away
                 const uint32_t first = it > kStages ? it - kStages : 0u;
                 for (uint32_t j = first; j < it; ++j)
-                    mbar_wait(&ctl->full[j % kStages], (j / kStages) & 1u, &ctl->drain_flag, 1000000ull);
+                    mbar_wait(&ctl->full[j % kStages], (j / kStages) & 1u, &ctl->drain_flag, kDrainLimitCycles);
             }
         }
         __syncwarp();
@@ -147,6 +147,8 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         // ------------------------------------------------------------ MMA issuer (one thread)
         if (elect_one()) {
             constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, false, false);
+            const uint64_t a_desc0 = make_smem_desc_sw128(smem_u32(smem_a), 16, 1024);
+            const uint64_t b_desc0 = make_smem_desc_sw128(smem_u32(smem_b), 16, 1024);
             uint32_t it = 0, tile_count = 0;
             bool ok = true;
             for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
@@ -166,14 +168,8 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                             break;
                         }
                         tc_fence_after_sync();
-                        const uint32_t a_addr = smem_u32(smem_a + stage * kABytes);
-                        const uint32_t b_addr = smem_u32(smem_b + stage * kBBytes);
-#pragma unroll
-                        for (int k = 0; k < kBK / 16; ++k) {
-                            umma_bf16_ss(d_tmem, make_smem_desc_sw128(a_addr + k * 32, 16, 1024),
-                                         make_smem_desc_sw128(b_addr + k * 32, 16, 1024), idesc,
-                                         (kb | k) != 0 ? 1u : 0u);
-                        }
+                        umma_ss_k64(d_tmem, a_desc0 + static_cast<uint64_t>(stage * (kABytes >> 4)),
+                                    b_desc0 + static_cast<uint64_t>(stage * (kBBytes >> 4)), idesc, kb != 0 ? 1u : 0u);
                         umma_commit(&ctl->empty[stage]);
                     }
                     if (ok) umma_commit(&ctl->tmem_full[acc]);
@@ -181,7 +177,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             }
             if (!ok) {
                 umma_commit(&ctl->drain);
-                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, 1000000ull);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, kDrainLimitCycles);
             }
         }
         __syncwarp();

@@ -10,18 +10,15 @@
 
 namespace rpx {
 
-// Upper bound for any single kernel-side wait.  A healthy wait lasts microseconds; when this
-// expires the kernel records RPX_ERR_TIMEOUT, drains what it has in flight and returns.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// Upper bound for any single kernel-side wait, in SM clock cycles (about 2-4 s between the
+// lowest and highest clocks of the part).  A healthy wait lasts microseconds; when this expires the
+// kernel records RPX_ERR_TIMEOUT, drains what it has in flight and returns.  The limit is kept on
+// the SM's own cycle counter: %globaltimer is far slower to read and must stay off the wait path.
+constexpr long long kWaitLimitCycles = 4000000000ll;
+constexpr long long kDrainLimitCycles = 2000000ll;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
 }
 
 __device__ __forceinline__ bool elect_one() {
@@ -68,17 +65,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the CTA-wide abort flag is (or becomes) set: the caller must
-// then leave its loop and fall through to the common teardown.
+// then leave its loop and fall through to the common teardown.  The first polls take no
+// timestamp at all; after that the cycle counter and the abort flag are checked every 32 polls.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint64_t limit_ns = kWaitLimitNs) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+                                          long long limit_cycles = kWaitLimitCycles) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     uint32_t polls = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++polls & 31u) == 0u) {
             if (*abort_flag != 0u) return false;
-            if (globaltimer_ns() - t0 > limit_ns) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1u;
                 return false;
             }
@@ -174,6 +174,68 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, u
         : "memory");
 }
 
+// ---- batched issue: one asm block per group of MMAs, so the single issuing thread spends about
+// three instructions per tcgen05.mma (descriptor add, add, mma) instead of rebuilding descriptors.
+// Descriptor offsets are in 16-byte units (the start-address field is the low 14 bits).
+#define RPX_UMMA_SS_STEP(off)                                                  \
+    "add.s64 da, %1, " #off ";\n"                                              \
+    "add.s64 db, %2, " #off ";\n"                                              \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n"
+#define RPX_UMMA_TS_STEP(acol, boff)                                           \
+    "add.u32 ta, %1, " #acol ";\n"                                             \
+    "add.s64 db, %2, " #boff ";\n"                                             \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n"
+
+// Four K=16 steps inside one 64-element (128-byte) swizzled K block: D (+)= A * B.
+__device__ __forceinline__ void umma_ss_k64(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate_first) {
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 pf, %4, 0;\n"
+        "setp.eq.b32 pt, %4, %4;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n" RPX_UMMA_SS_STEP(2) RPX_UMMA_SS_STEP(4)
+            RPX_UMMA_SS_STEP(6) "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+// Eight K=16 steps over two 64-element K blocks that lie 16 KiB (1024 units) apart: D = A * B.
+__device__ __forceinline__ void umma_ss_k128_overwrite(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 pf, %3, %3;\n"
+        "setp.eq.b32 pt, %3, %3;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n" RPX_UMMA_SS_STEP(2) RPX_UMMA_SS_STEP(4)
+            RPX_UMMA_SS_STEP(6) RPX_UMMA_SS_STEP(1024) RPX_UMMA_SS_STEP(1026) RPX_UMMA_SS_STEP(1028)
+                RPX_UMMA_SS_STEP(1030) "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+}
+// Four K=16 steps inside one 64-element K block: D = A * B (overwrite).
+__device__ __forceinline__ void umma_ss_k64_overwrite(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+    umma_ss_k64(tmem_d, adesc, bdesc, idesc, 0u);
+}
+// Eight K=16 steps of D (+)= A[tmem] * B[smem, MN-major]: A advances 8 TMEM columns (16 packed
+// bf16), B advances 16 rows of 128 bytes (128 units) per step.
+__device__ __forceinline__ void umma_ts_k128(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate_first) {
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 db;\n"
+        ".reg .b32 ta;\n"
+        "setp.ne.b32 pf, %4, 0;\n"
+        "setp.eq.b32 pt, %4, %4;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n" RPX_UMMA_TS_STEP(8, 128)
+            RPX_UMMA_TS_STEP(16, 256) RPX_UMMA_TS_STEP(24, 384) RPX_UMMA_TS_STEP(32, 512) RPX_UMMA_TS_STEP(40, 640)
+                RPX_UMMA_TS_STEP(48, 768) RPX_UMMA_TS_STEP(56, 896) "}\n" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+
 // 32 lanes x 32 columns of 32-bit: thread t of the warp receives columns c..c+31 of lane (base+t).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -233,16 +295,13 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t m, uint32_t n, b
            (static_cast<uint32_t>(b_mn_major) << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
+// exp2 on the special-function unit.  Written with the intrinsic rather than inline asm so that
+// the compiler sees its latency and can interleave independent elements.
+__device__ __forceinline__ float fast_exp2(float x) { return exp2f(x); }  // ex2.approx.ftz under --use_fast_math
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 }  // namespace rpx
