@@ -37,6 +37,10 @@ constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;
+#ifndef RPX_POLY_PAIRS_OF_4
+#define RPX_POLY_PAIRS_OF_4 1
+#endif
+constexpr int kPolyPairsOf4 = RPX_POLY_PAIRS_OF_4;  // of every 4 element pairs, how many take the polynomial exp2
 
 struct Ctl {
     uint64_t q_full;
@@ -438,21 +442,36 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 run_sum *= alpha;
                 run_max = new_max;
                 // ---- P = 2^(x - max) as packed bf16 pairs over the first 64 columns of S_t
-                const float neg_max = -run_max;
-                float part[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+                const uint64_t neg_max2 = f2_pack(-run_max, -run_max);
+                uint64_t part2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed accumulators = eight chains
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        const float e0 = fast_exp2(fmaf(__uint_as_float(sc[c][i]), p.scale_log2, neg_max));
-                        const float e1 = fast_exp2(fmaf(__uint_as_float(sc[c][i + 1]), p.scale_log2, neg_max));
-                        part[(i / 2) % 4] += e0 + e1;
+                        const uint64_t x = f2_fma(f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])),
+                                                  scale2, neg_max2);
+                        float e0, e1;
+                        if (((i / 2) % 4) < kPolyPairsOf4) {  // compile-time per unrolled pair
+                            poly_exp2_pair(x, e0, e1);
+                        } else {
+                            float x0, x1;
+                            f2_unpack(x, x0, x1);
+                            e0 = fast_exp2(x0);
+                            e1 = fast_exp2(x1);
+                        }
+                        part2[(i / 2) % 4] = f2_add(part2[(i / 2) % 4], f2_pack(e0, e1));
                         packed[i >> 1] = pack_bf16x2(e0, e1);
                     }
                     tmem_st16(my_s + half * 32 + c * 16, packed);
                 }
-                run_sum += (part[0] + part[1]) + (part[2] + part[3]);
+                {
+                    float a0, a1, b0, b1;
+                    f2_unpack(f2_add(f2_add(part2[0], part2[1]), f2_add(part2[2], part2[3])), a0, a1);
+                    (void)b0; (void)b1;
+                    run_sum += a0 + a1;
+                }
                 // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent until this warp's arrival
                 // below; each thread of the pair rescales its half of the row's O columns.  Done here,
                 // after the scores are dead, so the 32 staging registers do not force spills.

@@ -299,6 +299,58 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t m, uint32_t n, b
 // the compiler sees its latency and can interleave independent elements.
 __device__ __forceinline__ float fast_exp2(float x) { return exp2f(x); }  // ex2.approx.ftz under --use_fast_math
 
+// exp2 on the FMA/ALU pipes, for the share of elements taken off the special-function unit (16
+// results/clk/SM, as many cycles per attention tile as the tensor core needs for its two MMAs).
+// 2^x = 2^n * 2^f with n = round(x), f = x - n in [-0.5, 0.5]; 2^f by a degree-3 polynomial fitted
+// for minimum relative error (1.0e-4, against 2^-9 of the bf16 probabilities it feeds); 2^n is
+// added into the exponent field.  Inputs below -126 (masked scores are -inf) give a value < 2^-126.
+__device__ __forceinline__ float poly_exp2(float x) {
+    x = fmaxf(x, -126.f);
+    const float shifted = x + 12582912.f;  // 1.5 * 2^23: n lands in the low mantissa bits
+    const float n = shifted - 12582912.f;
+    const float f = x - n;
+    const float pf = fmaf(fmaf(fmaf(0.05500858f, f, 0.24221037f), f, 0.6932829f), f, 1.0f);
+    return __uint_as_float(__float_as_uint(pf) + (__float_as_uint(shifted) << 23));
+}
+
+// Packed fp32 pairs (sm_100 executes fma/add on two fp32 lanes of a 64-bit register per issue slot).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// poly_exp2 on a pair; see poly_exp2 for the method.
+__device__ __forceinline__ void poly_exp2_pair(uint64_t x, float& e0, float& e1) {
+    float x0, x1;
+    f2_unpack(x, x0, x1);
+    x = f2_pack(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t magic = f2_pack(12582912.f, 12582912.f), neg_magic = f2_pack(-12582912.f, -12582912.f);
+    const uint64_t shifted = f2_add(x, magic);
+    const uint64_t n = f2_add(shifted, neg_magic);
+    const uint64_t f = f2_fma(n, f2_pack(-1.f, -1.f), x);
+    uint64_t pf = f2_fma(f2_pack(0.05500858f, 0.05500858f), f, f2_pack(0.24221037f, 0.24221037f));
+    pf = f2_fma(pf, f, f2_pack(0.6932829f, 0.6932829f));
+    pf = f2_fma(pf, f, f2_pack(1.0f, 1.0f));
+    float p0, p1, s0, s1;
+    f2_unpack(pf, p0, p1);
+    f2_unpack(shifted, s0, s1);
+    e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(s0) << 23));
+    e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(s1) << 23));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
