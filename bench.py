@@ -271,15 +271,10 @@ def run_ours(args, rank, local_rank, world):
     sess.check_status()
     clocks = sampler.stop() if sampler else None
 
-    if world > 1:
-        tt = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(tt[0]), float(tt[1])
-        cnt = torch.tensor([wl.n_tokens, wl.n_suffix], dtype=torch.float64, device=dev)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        job_tokens, job_suffix = float(cnt[0]), float(cnt[1])
-    else:
-        job_tokens, job_suffix = float(wl.n_tokens), float(wl.n_suffix)
+    from paper_2608_14498_b200.dist import job_throughput
+
+    job_tokens, total_ms = job_throughput(wl.n_tokens, total_ms, dev)
+    job_suffix, e2e_ms = job_throughput(wl.n_suffix, e2e_ms, dev)
 
     if rank == 0:
         peaks = load_peaks()
@@ -321,6 +316,7 @@ def run_ours(args, rank, local_rank, world):
                     "h2d_bytes_per_step": hb.nbytes(), "d2h_bytes_per_step": (wl.n_prefix + wl.n_suffix) * 4,
                     "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": KERNELS_PER_SCORE * args.steps,
+            "gpu_launches_e2e": sess.kernels_last_host_pass * args.steps,
             "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
@@ -341,7 +337,7 @@ def run_ours(args, rank, local_rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))

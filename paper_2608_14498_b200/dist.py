@@ -1,0 +1,52 @@
+"""Multi-GPU plumbing for the scoring path: sequence sharding and whole-job timing.
+
+The path shards by sequence: every step (prefix attention, suffix attention, LM-head log-probs) is
+independent per sequence, W_vocab is replicated and each GPU owns its KV pool, so ranks never
+exchange data on the data path.  What is left for the host is (a) deciding which sequences a rank
+scores and (b) reducing per-rank timings and token counts to a job-level throughput.  Both work
+on any torch.distributed backend (NCCL on GPUs, gloo in the CPU tests).
+"""
+from __future__ import annotations
+
+from typing import List, Sequence, Tuple
+
+
+def sequence_cost(prompt_len: int, response_len: int, head_dim: int, num_q_heads: int, hidden: int, vocab: int) -> float:
+    """Algorithmic FLOPs of scoring one sequence (causal attention halves + LM head rows)."""
+    p, r = float(prompt_len), float(response_len)
+    attn = 2.0 * head_dim * num_q_heads * p * (p + 1) + 4.0 * head_dim * num_q_heads * (r * p + r * (r + 1) / 2)
+    lm = 2.0 * (p + r) * hidden * vocab
+    return attn + lm
+
+
+def partition_sequences(costs: Sequence[float], world_size: int) -> List[List[int]]:
+    """Longest-processing-time-first assignment of sequences to ranks.
+
+    Returns, per rank, the sorted indices of the sequences it scores.  Every sequence goes to
+    exactly one rank; the heaviest rank carries at most 4/3 of the optimum (the LPT bound)."""
+    if world_size <= 0:
+        raise ValueError("world_size must be positive")
+    load = [0.0] * world_size
+    parts: List[List[int]] = [[] for _ in range(world_size)]
+    for idx in sorted(range(len(costs)), key=lambda i: (-costs[i], i)):
+        r = min(range(world_size), key=lambda k: (load[k], k))
+        parts[r].append(idx)
+        load[r] += float(costs[idx])
+    return [sorted(p) for p in parts]
+
+
+def job_throughput(local_units: float, local_ms: float, device=None) -> Tuple[float, float]:
+    """(units of all ranks, max over ranks of the elapsed milliseconds).
+
+    Collective-free on the data path; this is the only exchange of a run and it carries two
+    numbers.  Without an initialised process group it returns the local values."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(local_units), float(local_ms)
+    t = torch.tensor([float(local_ms)], dtype=torch.float64, device=device)
+    n = torch.tensor([float(local_units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(n.item()), float(t.item())

@@ -68,6 +68,9 @@ class ScoringSession:
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self._ws = {}
         self._staging: Optional[Batch] = None
+        self._copy_stream = None
+        self._staging_free = None
+        self.kernels_last_host_pass = 0
         self._out = {}
 
     def _workspace(self, key: str, nbytes: int):
@@ -123,19 +126,75 @@ class ScoringSession:
         mark(4)
         return lp_p, lp_s, o_p, o_s
 
-    def score_from_host(self, hb: Batch, lp_p_host, lp_s_host):
-        """Pinned host batch in, log-probs out into the pinned ``lp_*_host`` tensors.  Copies and
-        kernels are enqueued on the current stream; the caller synchronises."""
+    def score_from_host(self, hb: Batch, lp_p_host, lp_s_host, lm_slices: int = 4):
+        """Pinned host batch in, log-probs out into the pinned ``lp_*_host`` tensors.
+
+        Host->device copies run on a copy stream in the order the kernels need them and each
+        kernel waits only for its own inputs: the prompt rows of the LM head (the longest kernel)
+        are cut into ``lm_slices`` row slices so that scoring starts after the first slice has
+        landed and the remaining copies hide behind it.  Kernels and the device->host copy of the
+        results are enqueued on the current stream; the caller synchronises."""
         t = self.torch
         if self._staging is None or any(tuple(a.shape) != tuple(c.shape) or a.dtype != c.dtype
                                         for a, c in zip(self._staging.tensors(), hb.tensors())):
             dev = [t.empty(x.shape, dtype=x.dtype, device=self.device) for x in hb.tensors()]
             self._staging = Batch(*dev, hb.max_prefix_len, hb.max_suffix_len)
-        for dst, src in zip(self._staging.tensors(), hb.tensors()):
-            dst.copy_(src, non_blocking=True)
-        lp_p, lp_s, _, _ = self.score(self._staging)
+            self._copy_stream = t.cuda.Stream(device=self.device)
+            self._staging_free = None
+        d = self._staging
+        main = t.cuda.current_stream()
+        copy = self._copy_stream
+        if self._staging_free is not None:
+            copy.wait_event(self._staging_free)  # last pass has finished reading the staging buffers
+        else:
+            copy.wait_stream(main)
+
+        def upload(pairs):
+            with t.cuda.stream(copy):
+                for dst, src in pairs:
+                    dst.copy_(src, non_blocking=True)
+                ev = t.cuda.Event()
+                ev.record(copy)
+            return ev
+
+        n_p = hb.hidden_p.shape[0]
+        bounds = [n_p * i // lm_slices for i in range(lm_slices + 1)] if n_p > 0 else [0, 0]
+        ev_ids = upload([(d.ids_p, hb.ids_p)])
+        ev_slices = [upload([(d.hidden_p[a:b], hb.hidden_p[a:b])]) for a, b in zip(bounds[:-1], bounds[1:])]
+        ev_prefix = upload([(d.q_p, hb.q_p), (d.k_p, hb.k_p), (d.v_p, hb.v_p), (d.cu_prefix, hb.cu_prefix),
+                            (d.block_table, hb.block_table)])
+        ev_suffix = upload([(d.q_s, hb.q_s), (d.k_s, hb.k_s), (d.v_s, hb.v_s), (d.cu_suffix, hb.cu_suffix),
+                            (d.prefix_lens, hb.prefix_lens), (d.hidden_s, hb.hidden_s), (d.ids_s, hb.ids_s)])
+
+        cache = (self.k_cache, self.v_cache, d.block_table)
+        code = B._dtype_code(d.hidden_p)
+        vocab, hdim = self.w_vocab.shape
+        lp_p = self._buf("lp_p", (n_p,), t.float32)
+        lp_s = self._buf("lp_s", (hb.hidden_s.shape[0],), t.float32)
+        o_p = self._buf("o_p", d.q_p.shape, d.q_p.dtype)
+        o_s = self._buf("o_s", d.q_s.shape, d.q_s.dtype)
+        lm_ws = self._workspace("lm", B.token_logprobs_workspace_bytes(max(n_p, hb.hidden_s.shape[0]), hdim, vocab, code))
+        attn_ws = self._workspace("attn", max(
+            B.prefix_attn_workspace_bytes(d.q_p.shape[1], d.k_p.shape[1], d.q_p.shape[2], B._dtype_code(d.q_p), d.q_p.shape[0]),
+            B.suffix_attn_workspace_bytes(d.q_s.shape[1], d.k_s.shape[1], d.q_s.shape[2], B._dtype_code(d.q_s), d.q_s.shape[0])))
+        main.wait_event(ev_ids)
+        for (a, b), ev in zip(zip(bounds[:-1], bounds[1:]), ev_slices):
+            main.wait_event(ev)
+            if b > a:
+                B.token_logprobs(d.hidden_p[a:b], self.w_vocab, d.ids_p[a:b], logprobs=lp_p[a:b], workspace=lm_ws,
+                                 device_status=self.status)
+        main.wait_event(ev_prefix)
+        B.prefix_attn(d.q_p, d.k_p, d.v_p, d.cu_prefix, d.max_prefix_len, cache=cache, out=o_p, workspace=attn_ws,
+                      device_status=self.status)
+        main.wait_event(ev_suffix)
+        B.suffix_attn(d.q_s, d.k_s, d.v_s, d.cu_suffix, d.prefix_lens, d.max_suffix_len, d.max_prefix_len, cache=cache,
+                      out=o_s, workspace=attn_ws, device_status=self.status)
+        B.token_logprobs(d.hidden_s, self.w_vocab, d.ids_s, logprobs=lp_s, workspace=lm_ws, device_status=self.status)
+        self._staging_free = t.cuda.Event()
+        self._staging_free.record(main)
         lp_p_host.copy_(lp_p, non_blocking=True)
         lp_s_host.copy_(lp_s, non_blocking=True)
+        self.kernels_last_host_pass = 2 + 2 * (sum(1 for a, b in zip(bounds[:-1], bounds[1:]) if b > a) + 1)
         return lp_p_host, lp_s_host
 
     def check_status(self) -> None:

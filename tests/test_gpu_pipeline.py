@@ -1,0 +1,48 @@
+"""The scoring session: device-resident pass vs the overlapped host-resident pass vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_14498_b200 import workloads as wk
+from paper_2608_14498_b200.pipeline import Batch, ScoringSession
+from helpers import to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _host_batch(wl):
+    def t(a):
+        x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return x.pin_memory()
+
+    pre, suf = wl.prefix_rows(), wl.suffix_rows()
+    return Batch(t(wl.q[pre]), t(wl.k[pre]), t(wl.v[pre]), t(wl.q[suf]), t(wl.k[suf]), t(wl.v[suf]), t(wl.cu_prefix),
+                 t(wl.cu_suffix), t(wl.prompt_lens), t(wl.block_table), t(wl.hidden[pre]), t(wl.ids[pre]),
+                 t(wl.hidden[suf]), t(wl.ids[suf]), int(wl.prompt_lens.max()), int(wl.response_lens.max()))
+
+
+def test_host_pass_equals_device_pass_and_oracle(cuda_device):
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 3, 4, 2, 128, 512, 6000, ("list", [700, 130, 257]), ("list", [90, 300, 129]))
+    wl = wk.make_workload(cfg, seed=31)
+    hb = _host_batch(wl)
+    db = Batch(*[x.to(dev) for x in hb.tensors()], hb.max_prefix_len, hb.max_suffix_len)
+    sess = ScoringSession(to_device(wl.w, dev), wl.num_blocks, cfg.num_kv_heads, cfg.head_dim)
+    lp_p, lp_s, o_p, o_s = sess.score(db)
+    lp_p, lp_s, o_p, o_s = lp_p.clone(), lp_s.clone(), o_p.clone(), o_s.clone()
+    host_p = torch.empty(wl.n_prefix, dtype=torch.float32).pin_memory()
+    host_s = torch.empty(wl.n_suffix, dtype=torch.float32).pin_memory()
+    for _ in range(2):  # the second pass reuses the staging buffers while the first may still be in flight
+        sess.score_from_host(hb, host_p, host_s, lm_slices=3)
+    torch.cuda.synchronize()
+    sess.check_status()
+    assert torch.equal(host_p, lp_p.cpu()) and torch.equal(host_s, lp_s.cpu())
+    assert torch.equal(sess._out["o_p"], o_p) and torch.equal(sess._out["o_s"], o_s)
+    assert sess.kernels_last_host_pass == 2 + 2 * 4
+    # against the oracle: concatenated prefix and suffix log-probs are the full-sequence values
+    ref, _ = oracle.logprob_rows(wl.hidden, wl.w, wl.ids)
+    got = np.empty(wl.n_tokens)
+    got[wl.prefix_rows()] = host_p.double().numpy()
+    got[wl.suffix_rows()] = host_s.double().numpy()
+    assert np.abs(got - ref).max() <= 5e-4
