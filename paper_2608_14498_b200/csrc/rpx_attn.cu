@@ -4,14 +4,13 @@
 // One CTA owns two adjacent 128-row query tiles of one (sequence, query head) and walks the key
 // tiles (128 keys) that those rows may see: first the cached prefix tiles (suffix pass only,
 // unmasked except the last partial one), then the self tiles up to each query tile's diagonal.
-//   warps 0-7  : softmax of query tile 0: warp w owns rows 32*(w%4).. (its TMEM lane quarter) and
-//                key columns 64*(w/4)..+63, so two threads share a row and twice as many warps
-//                hide each other's latencies; the pair exchanges its row maximum (and, at the
-//                end, its row sum) through shared memory and a 64-thread mbarrier
-//   warps 8-15 : softmax of query tile 1
-//   warp  16   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
+//   warps 0-3 : softmax of query tile 0: thread = one row = one TMEM lane, all 128 scores of the
+//               row in registers (two threads per row were tried: the extra exchange of the row
+//               maximum cost more than the shorter dependency chains gained)
+//   warps 4-7 : softmax of query tile 1
+//   warp  8   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
 //               16-token page); it also stores the diagonal K/V tiles into the paged cache
-//   warp  17   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
+//   warp  9   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
 //               O_t += P_t V  (P_t = bf16 probabilities written back into the first 64 columns
 //               of S_t's TMEM region and consumed as the TMEM A operand; V straight from its
 //               [keys][d] tile as an MN-major B operand)
@@ -31,8 +30,10 @@ namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
 constexpr int kSlots = 5;
-constexpr int kThreads = 576;
-constexpr int kProducerWarp = 16, kMmaWarp = 17;
+constexpr int kChunks = kTileK / 32;  // 32-column TMEM loads per row and step
+constexpr int kWarpsPerTile = 4;
+constexpr int kProducerWarp = 2 * kWarpsPerTile, kMmaWarp = kProducerWarp + 1;
+constexpr int kThreads = 32 * (kMmaWarp + 1);
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -49,13 +50,11 @@ struct Ctl {
     uint64_t s_full[2];   // tensor core -> softmax: S_t(j) is in TMEM (and PV_t(j-1) has finished)
     uint64_t p_ready[2];  // softmax -> tensor core: P_t(j) is in TMEM, O_t rescaled if needed
     uint64_t o_done[2];   // tensor core -> softmax: the last PV_t has finished
-    uint64_t pair_sync[2][4];  // the two warps sharing rows 32q..32q+31 of tile t
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t drain_flag;
     uint32_t data_error;
-    float xchg[2][2][128];     // [tile][column half][row]: row maximum, later row sum
 };
 
 template <int D>
@@ -137,9 +136,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&ctl->s_full[t], 1);
-            mbar_init(&ctl->p_ready[t], 8);  // one arrival per softmax warp
+            mbar_init(&ctl->p_ready[t], kWarpsPerTile);  // one arrival per softmax warp
             mbar_init(&ctl->o_done[t], 1);
-            for (int q = 0; q < 4; ++q) mbar_init(&ctl->pair_sync[t][q], 2);  // one arrival per warp of the pair
         }
         mbar_init(&ctl->drain, 1);
         ctl->abort_flag = 0;
@@ -369,16 +367,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         __syncwarp();
     } else {
         // =========================================================== softmax warps
-        const int t = warp >> 3;
+        const int t = warp / kWarpsPerTile;
         if (t == 0 || active1) {
             const uint32_t quarter = warp & 3;
-            const int half = (warp >> 2) & 1;
             const int32_t row = quarter * 32 + lane;
             const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
             const uint32_t lane_addr = (quarter * 32u) << 16;
-            uint64_t* pair_bar = &ctl->pair_sync[t][quarter];
-            float* my_slot = &ctl->xchg[t][half][row];
-            const float* peer_slot = &ctl->xchg[t][half ^ 1][row];
             const int32_t my_tiles = n_tile0 + t;
             const uint32_t my_s = tmem_base + t * 128 + lane_addr;        // this thread's lane of S_t / P_t
             const uint32_t my_o = tmem_base + 256 + t * 128 + lane_addr;  // and of O_t
@@ -390,12 +384,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     break;
                 }
                 tc_fence_after_sync();
-                // ---- this thread's 64 scores of the row
-                uint32_t sc[2][32];
+                // ---- the row's 128 scores
+                uint32_t sc[kChunks][32];
 #pragma unroll
-                for (int c = 0; c < 2; ++c) tmem_ld32(my_s + half * 64 + c * 32, sc[c]);
+                for (int c = 0; c < kChunks; ++c) tmem_ld32(my_s + c * 32, sc[c]);
                 tmem_ld_wait();
-                // ---- how many leading keys of this tile the row may see, counted from this half
+                // ---- how many leading keys of this tile the row may see
                 int32_t n_vis;
                 if (j < n_prefix_tiles) {
                     n_vis = min(kTileK, len_p - j * kTileK);
@@ -403,10 +397,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     const int32_t jt = j - n_prefix_tiles;
                     n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
                 }
-                n_vis -= half * 64;
-                if (n_vis < 64) {
+                if (n_vis < kTileK) {
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
+                    for (int c = 0; c < kChunks; ++c)
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (c * 32 + i >= n_vis) sc[c][i] = 0xff800000u;  // -inf
@@ -416,25 +409,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
 #pragma unroll
                 for (int u = 0; u < 8; ++u) mx[u] = -CUDART_INF_F;
 #pragma unroll
-                for (int c = 0; c < 2; ++c)
+                for (int c = 0; c < kChunks; ++c)
 #pragma unroll
                     for (int i = 0; i < 32; i += 8)
 #pragma unroll
                         for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(sc[c][i + u]));
                 float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                                    fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                // ---- agree on the row maximum with the thread that holds the other 64 columns.  The
-                // barrier also orders both threads' S loads before either thread's P stores, which
-                // land on columns the other thread reads its scores from.
-                *my_slot = cmax;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(pair_bar);  // a warp-wide arrival: 256 single arrivals per step
-                                                       // would serialise on the barrier word
-                if (!mbar_wait(pair_bar, j & 1, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                cmax = fmaxf(cmax, *peer_slot) * p.scale_log2;  // scale > 0, so max commutes with the scaling
+                cmax *= p.scale_log2;  // scale > 0, so max commutes with the scaling
                 const bool grow = cmax > run_max + kRescaleThreshold;
                 const float new_max = grow ? cmax : run_max;
                 const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
@@ -446,25 +428,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const uint64_t neg_max2 = f2_pack(-run_max, -run_max);
                 uint64_t part2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed accumulators = eight chains
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
+                for (int c = 0; c < kChunks; ++c) {
                     uint32_t packed[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
                         const uint64_t x = f2_fma(f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])),
                                                   scale2, neg_max2);
                         float e0, e1;
+                        float x0, x1;
+                        f2_unpack(x, x0, x1);
                         if (((i / 2) % 4) < kPolyPairsOf4) {  // compile-time per unrolled pair
-                            poly_exp2_pair(x, e0, e1);
+                            e0 = poly_exp2(x0);  // scalar form: its constants are immediates, the packed
+                            e1 = poly_exp2(x1);  // form would pin seven register pairs in this loop
                         } else {
-                            float x0, x1;
-                            f2_unpack(x, x0, x1);
                             e0 = fast_exp2(x0);
                             e1 = fast_exp2(x1);
                         }
                         part2[(i / 2) % 4] = f2_add(part2[(i / 2) % 4], f2_pack(e0, e1));
                         packed[i >> 1] = pack_bf16x2(e0, e1);
                     }
-                    tmem_st16(my_s + half * 32 + c * 16, packed);
+                    tmem_st16(my_s + c * 16, packed);
                 }
                 {
                     float a0, a1, b0, b1;
@@ -473,13 +456,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     run_sum += a0 + a1;
                 }
                 // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent until this warp's arrival
-                // below; each thread of the pair rescales its half of the row's O columns.  Done here,
+                // below.  Done here,
                 // after the scores are dead, so the 32 staging registers do not force spills.
                 if (rescale) {
 #pragma unroll 1
-                    for (int c = 0; c < D / 64; ++c) {
+                    for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
-                        const uint32_t addr = my_o + half * (D / 2) + c * 32;
+                        const uint32_t addr = my_o + c * 32;
                         tmem_ld32(addr, r);
                         tmem_ld_wait();
 #pragma unroll
@@ -492,26 +475,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->p_ready[t]);
             }
-            // ---- epilogue: O / l -> global, LSE; each thread of the pair writes half of the row
+            // ---- epilogue: O / l -> global, LSE
             if (ok) ok = mbar_wait(&ctl->o_done[t], 0, abort_flag);
             if (ok) {
-                // the last PV ran after every thread's last p_ready arrival, hence after the partner
-                // read this thread's last maximum: the slot can now carry the row sum
-                *my_slot = run_sum;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(pair_bar);
-                ok = mbar_wait(pair_bar, my_tiles & 1, abort_flag);
-            }
-            if (ok) {
                 tc_fence_after_sync();
-                run_sum += *peer_slot;
                 const bool row_valid = q_local < len_q;
                 const float inv = 1.f / run_sum;
-                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D + half * (D / 2);
+                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
 #pragma unroll 1
-                for (int c = 0; c < D / 64; ++c) {
+                for (int c = 0; c < D / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld32(my_o + half * (D / 2) + c * 32, r);
+                    tmem_ld32(my_o + c * 32, r);
                     tmem_ld_wait();
                     if (row_valid) {
                         if (p.out_f32) {
@@ -534,7 +508,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         }
                     }
                 }
-                if (half == 0 && row_valid && p.lse != nullptr)
+                if (row_valid && p.lse != nullptr)
                     p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
             }
         }
