@@ -52,11 +52,13 @@ struct LogprobArgs {
     int32_t hidden_dim, vocab;
     float* logprobs;
     float* lse;
-    void* partials;       // float4 [logprob_num_chunks(vocab)][n_tokens]
+    void* partials;       // float4 [logprob_num_chunks(vocab, tiles_per_chunk)][n_tokens]
+    int32_t tiles_per_chunk;  // vocabulary tiles (256 columns) one work item sweeps
     int32_t* device_status;
     cudaStream_t stream;
 };
-int32_t logprob_num_chunks(int32_t vocab);
+int32_t logprob_tiles_per_chunk(int64_t n_tokens);  // the default policy
+int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk);
 rpx_status_t launch_token_logprobs(const LogprobArgs& a);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

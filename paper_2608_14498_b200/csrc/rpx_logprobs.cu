@@ -2,8 +2,8 @@
 //
 //   logprob[n] = z[n, target[n]] - ln sum_v exp(z[n, v]),   z = hidden . W_vocab^T  (never stored)
 //
-// One persistent CTA per SM.  A work item is (row tile of 128 rows, chunk of kTilesPerChunk vocab
-// tiles of 256 columns): the CTA sweeps the chunk tile by tile; each tile is a TMA-fed tcgen05
+// One persistent CTA per SM.  A work item is (row tile of 128 rows, chunk of 16 (4 for small row
+// counts) vocab tiles of 256 columns): the CTA sweeps the chunk tile by tile; each tile is a TMA-fed tcgen05
 // GEMM over the hidden dimension into one of two 128x256 fp32 TMEM accumulators, and while the
 // tensor core fills one accumulator the four epilogue warps fold the other into a running
 // (max, sum-exp, target-logit) per row.  One partial per (chunk, row) goes to the workspace; a
@@ -25,7 +25,9 @@ namespace rpx {
 namespace {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
-constexpr int kTilesPerChunk = 16;
+constexpr int kTilesPerChunkLarge = 16;  // many row tiles: long items, few partial records
+constexpr int kTilesPerChunkSmall = 4;   // few row tiles: short items, so the last wave is short too
+constexpr int kSmallRowTiles = 64;
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
@@ -51,6 +53,7 @@ struct Params {
     int32_t n_row_tiles;
     int32_t n_vocab_tiles;
     int32_t n_chunks;
+    int32_t tiles_per_chunk;
     int32_t group_width;   // vocab chunks in flight side by side
     int32_t total_items;
     const int32_t* target_ids;
@@ -71,8 +74,8 @@ __device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
     Item it;
     it.m_tile = rem / width;
     it.chunk = first + rem % width;
-    it.tile_begin = it.chunk * kTilesPerChunk;
-    it.tile_end = min(it.tile_begin + kTilesPerChunk, p.n_vocab_tiles);
+    it.tile_begin = it.chunk * p.tiles_per_chunk;
+    it.tile_end = min(it.tile_begin + p.tiles_per_chunk, p.n_vocab_tiles);
     return it;
 }
 
@@ -284,9 +287,13 @@ __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int3
 
 }  // namespace
 
-int32_t logprob_num_chunks(int32_t vocab) {
+int32_t logprob_tiles_per_chunk(int64_t n_tokens) {
+    return (n_tokens + kBM - 1) / kBM <= kSmallRowTiles ? kTilesPerChunkSmall : kTilesPerChunkLarge;
+}
+
+int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk) {
     const int32_t tiles = (vocab + kBN - 1) / kBN;
-    return (tiles + kTilesPerChunk - 1) / kTilesPerChunk;
+    return (tiles + tiles_per_chunk - 1) / tiles_per_chunk;
 }
 
 rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
@@ -310,7 +317,8 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     p.k_blocks = (a.hidden_dim + kBK - 1) / kBK;
     p.n_row_tiles = static_cast<int32_t>((a.n_tokens + kBM - 1) / kBM);
     p.n_vocab_tiles = (a.vocab + kBN - 1) / kBN;
-    p.n_chunks = logprob_num_chunks(a.vocab);
+    p.tiles_per_chunk = a.tiles_per_chunk;
+    p.n_chunks = logprob_num_chunks(a.vocab, a.tiles_per_chunk);
     const int64_t total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
     if (total > INT32_MAX) return RPX_ERR_SHAPE;
     p.total_items = static_cast<int32_t>(total);
@@ -387,7 +395,7 @@ extern "C" RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, in
     if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0 || (reinterpret_cast<uintptr_t>(w_vocab) & 15u) != 0)
         return RPX_ERR_ALIGN;
     // one 16-byte record per (vocab chunk, row) must fit in the built-in array
-    const size_t need = static_cast<size_t>(logprob_num_chunks(vocab)) * static_cast<size_t>(n_tokens) * sizeof(float4);
+    const size_t need = static_cast<size_t>(logprob_num_chunks(vocab, kTilesPerChunkLarge)) * static_cast<size_t>(n_tokens) * sizeof(float4);
     if (need > static_cast<size_t>(RPX_STATIC_SCRATCH_BYTES)) return RPX_ERR_WORKSPACE;
     if (rpx_status_t rc = check_arch()) return rc;
     void* scratch = nullptr;
@@ -404,6 +412,7 @@ extern "C" RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, in
     a.logprobs = logprobs;
     a.lse = lse;
     a.partials = scratch;
+    a.tiles_per_chunk = kTilesPerChunkLarge;  // the documented size limit assumes 16-tile chunks
     a.device_status = device_status;
     a.stream = static_cast<cudaStream_t>(cuda_stream);
     return launch_token_logprobs(a);

@@ -173,7 +173,8 @@ class ScoringSession:
         lp_s = self._buf("lp_s", (hb.hidden_s.shape[0],), t.float32)
         o_p = self._buf("o_p", d.q_p.shape, d.q_p.dtype)
         o_s = self._buf("o_s", d.q_s.shape, d.q_s.dtype)
-        lm_ws = self._workspace("lm", B.token_logprobs_workspace_bytes(max(n_p, hb.hidden_s.shape[0]), hdim, vocab, code))
+        lm_calls = [b - a for a, b in zip(bounds[:-1], bounds[1:])] + [hb.hidden_s.shape[0]]
+        lm_ws = self._workspace("lm", max(B.token_logprobs_workspace_bytes(n, hdim, vocab, code) for n in lm_calls))
         attn_ws = self._workspace("attn", max(
             B.prefix_attn_workspace_bytes(d.q_p.shape[1], d.k_p.shape[1], d.q_p.shape[2], B._dtype_code(d.q_p), d.q_p.shape[0]),
             B.suffix_attn_workspace_bytes(d.q_s.shape[1], d.k_s.shape[1], d.q_s.shape[2], B._dtype_code(d.q_s), d.q_s.shape[0])))

@@ -47,7 +47,8 @@ def test_workspace_arithmetic(lib):
     # 152064 columns = 594 tiles of 256 = 38 chunks of 16 tiles; one float4 per (chunk, row)
     assert B.token_logprobs_workspace_bytes(34816, 3584, 152064, B.RPX_BF16) == 38 * 34816 * 16
     f32 = B.token_logprobs_workspace_bytes(288, 256, 4096, B.RPX_F32)
-    assert f32 == 1 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
+    # up to 64 row tiles the chunks are 4 vocabulary tiles long: 4096 columns = 16 tiles = 4 chunks
+    assert f32 == 4 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
     assert B.token_logprobs_workspace_bytes(0, 256, 4096, B.RPX_BF16) == 0
 
 
