@@ -39,9 +39,10 @@ if ROOT not in sys.path:
 from paper_2608_14498_b200 import workloads as wk  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (read + write) of one LM-head partial-kernel launch on the bench workload, scaled from
-# an ncu capture of a smaller launch of the same kernel; see profiles/.  None until captured.
-LM_HEAD_TRAFFIC_BYTES = None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the LM-head partial kernel on the
+# benchmark's prompt-row launch (32768 x 152064 x 3584), from a one-pass ncu capture of this very
+# command; summary in profiles/lm_head_partial_kernel__slice_8192x32768x3584.md.  Other configs: None.
+LM_HEAD_TRAFFIC_BYTES = {"C2": 11.40e9 + 24.0e6}
 
 
 def load_peaks():
@@ -310,7 +311,7 @@ def run_ours(args, rank, local_rank, world):
                          "bound": "tensor", "achieved": lm_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": lm_tf / peak_tf,
                          "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
                          "frac_of_burst_peak": lm_tf / float(peaks["bf16_tflops"]),
-                         "traffic": LM_HEAD_TRAFFIC_BYTES,
+                         "traffic": LM_HEAD_TRAFFIC_BYTES.get(args.config),
                          "algorithmic_bytes": (wl.n_prefix * cfg.hidden + cfg.vocab * cfg.hidden) * 2 + 8 * wl.n_prefix},
             "e2e": {"value": job_tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s",
                     "h2d_bytes_per_step": hb.nbytes(), "d2h_bytes_per_step": (wl.n_prefix + wl.n_suffix) * 4,
