@@ -179,6 +179,15 @@ RPX_API size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int6
 RPX_API size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
                                           rpx_dtype_t dtype);
 
+/*
+ * Self-test of the bounded kernel-side wait every kernel of this library relies on (no counterpart
+ * in the paper).  Enqueues a one-CTA kernel in which one thread waits, for at most `limit_cycles`
+ * SM cycles (1 .. 2e9), on a barrier that nothing ever signals; the wait must give up, the kernel
+ * must return, and RPX_ERR_TIMEOUT must appear in *device_status (device int32, zeroed by the
+ * caller).  The CUDA context stays usable: nothing traps, faults or spins without a limit.
+ */
+RPX_API rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* device_status, void* cuda_stream);
+
 /* Static string for a status code; never NULL. */
 RPX_API const char* rpx_status_string(rpx_status_t status);
 

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     load_library,
     prefix_attn,
     prefix_attn_workspace_bytes,
+    selftest_bounded_wait,
     status_string,
     suffix_attn,
     suffix_attn_workspace_bytes,

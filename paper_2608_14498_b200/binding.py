@@ -26,6 +26,7 @@ EXPORTS = (
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
     "rpx_token_logprobs_workspace_bytes",
+    "rpx_selftest_bounded_wait",
     "rpx_status_string",
     "rpx_version",
 )
@@ -90,6 +91,8 @@ def load_library():
     lib.rpx_suffix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
     lib.rpx_token_logprobs_workspace_bytes.restype = sz
     lib.rpx_token_logprobs_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    lib.rpx_selftest_bounded_wait.restype = i32
+    lib.rpx_selftest_bounded_wait.argtypes = [i64, vp, vp]
     lib.rpx_status_string.restype = ctypes.c_char_p
     lib.rpx_status_string.argtypes = [i32]
     lib.rpx_version.restype = i32
@@ -179,6 +182,13 @@ def suffix_attn_workspace_bytes(num_q_heads, num_kv_heads, head_dim, dtype_code,
 def token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype_code) -> int:
     return int(load_library().rpx_token_logprobs_workspace_bytes(int(n_tokens), int(hidden_dim), int(vocab),
                                                                  int(dtype_code)))
+
+
+def selftest_bounded_wait(limit_cycles: int, device_status, stream=None) -> None:
+    """rpx_selftest_bounded_wait: a wait that must time out and report RPX_ERR_TIMEOUT in device_status."""
+    rc = load_library().rpx_selftest_bounded_wait(int(limit_cycles), _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_selftest_bounded_wait")
 
 
 # ------------------------------------------------------------------ the three calls

@@ -196,6 +196,13 @@ rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, c
     return launch_token_logprobs(a);
 }
 
+rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* device_status, void* cuda_stream) {
+    if (device_status == nullptr) return RPX_ERR_NULL;
+    if (limit_cycles <= 0 || limit_cycles > 2000000000ll) return RPX_ERR_SHAPE;
+    if (rpx_status_t rc = check_arch()) return rc;
+    return launch_bounded_wait_selftest(limit_cycles, device_status, static_cast<cudaStream_t>(cuda_stream));
+}
+
 const char* rpx_status_string(rpx_status_t status) {
     switch (status) {
         case RPX_OK: return "ok";

@@ -5,6 +5,7 @@
 #include <mutex>
 
 #include "rpx_internal.h"
+#include "rpx_ptx.cuh"
 
 namespace rpx {
 
@@ -37,7 +38,28 @@ __global__ void cast_f32_bf16_kernel(const float* __restrict__ src, int64_t src_
     }
 }
 
+// One thread waits on an mbarrier nobody arrives on, so the bounded wait has to run out.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, int32_t* status) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool completed = mbar_wait(&bar, 0, &abort_flag, limit_cycles);
+        if (!completed && abort_flag != 0u && status != nullptr) atomicCAS(status, 0, RPX_ERR_TIMEOUT);
+    }
+}
+
 }  // namespace
+
+rpx_status_t launch_bounded_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t stream) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(limit_cycles, status);
+    return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
+}
 
 rpx_status_t encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                               const uint64_t* strides_bytes, const uint32_t* box) {

@@ -61,6 +61,8 @@ int32_t logprob_tiles_per_chunk(int64_t n_tokens);  // the default policy
 int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk);
 rpx_status_t launch_token_logprobs(const LogprobArgs& a);
 
+rpx_status_t launch_bounded_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t stream);
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace rpx
