@@ -335,6 +335,67 @@ def run_ours(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def run_group(args):
+    """Prompt groups (GRPO: N sampled responses per prompt).  Times one scoring pass with the prompt
+    prefix computed once per group (cache rows aliased by the group's members) against the same
+    members scored as unrelated sequences, each with its own copy of the prompt."""
+    import torch
+
+    import paper_2608_14498_b200 as rpx
+    from paper_2608_14498_b200.pipeline import Batch, ScoringSession
+
+    dev = torch.device("cuda", 0)
+    cfg = wk.CONFIGS[args.config]
+    gw = wk.make_group_workload(cfg, args.group, seed=0)
+    pro, mem = gw.prompts, gw.members
+
+    def t(a):
+        x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return x.to(dev)
+
+    w = t(pro.w)
+    sess = ScoringSession(w, pro.num_blocks, cfg.num_kv_heads, cfg.head_dim)
+    pre, suf = mem.prefix_rows(), mem.suffix_rows()
+    shared = Batch(t(pro.q), t(pro.k), t(pro.v), t(mem.q[suf]), t(mem.k[suf]), t(mem.v[suf]), t(pro.cu_full),
+                   t(mem.cu_suffix), t(mem.prompt_lens), t(gw.member_table), t(pro.hidden), t(pro.ids), t(mem.hidden[suf]),
+                   t(mem.ids[suf]), int(pro.prompt_lens.max()), int(mem.response_lens.max()))
+    own_table, own_blocks = wk.make_block_table(mem.prompt_lens, seed=1)
+    sess_own = ScoringSession(w, own_blocks, cfg.num_kv_heads, cfg.head_dim)
+    unshared = Batch(t(mem.q[pre]), t(mem.k[pre]), t(mem.v[pre]), shared.q_s, shared.k_s, shared.v_s, t(mem.cu_prefix),
+                     shared.cu_suffix, shared.prefix_lens, t(own_table), t(mem.hidden[pre]), t(mem.ids[pre]), shared.hidden_s,
+                     shared.ids_s, shared.max_prefix_len, shared.max_suffix_len)
+
+    def timed(session, batch):
+        for _ in range(3):
+            session.score(batch)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            session.score(batch)
+        e1.record()
+        torch.cuda.synchronize()
+        session.check_status()
+        return e0.elapsed_time(e1) / args.steps
+
+    ms_shared, ms_unshared = timed(sess, shared), timed(sess_own, unshared)
+    lp_a = sess.score(shared)[1].clone()
+    lp_b = sess_own.score(unshared)[1]
+    torch.cuda.synchronize()
+    line = {
+        "metric": "scored_tokens_per_s", "value": mem.n_tokens / (ms_shared * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": 3, "ms_per_step": ms_shared, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} as {cfg.batch} prompts x {args.group} responses, prefix scored once per prompt",
+                   "member_tokens": mem.n_tokens, "prompt_rows_computed": pro.n_tokens, "response_rows": mem.n_suffix},
+        "group": {"size": args.group, "ms_shared_prefix": ms_shared, "ms_every_member_own_prefix": ms_unshared,
+                  "speedup": ms_unshared / ms_shared,
+                  "suffix_logprob_max_abs_diff": float((lp_a - lp_b).abs().max().item())},
+        "gpu_launches": 6 * args.steps,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -345,11 +406,15 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=48, help="tokens the oracle scores for cpu_baseline")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--group", type=int, default=0, help="score prompt groups of this size (prefix once per prompt)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.group > 0:
+        if rank == 0:
+            run_group(args)
+    elif args.impl == "reference":
         run_reference(args, rank)
     else:
         run_ours(args, rank, local_rank, world)

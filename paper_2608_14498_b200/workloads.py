@@ -270,3 +270,51 @@ def sample_logprob_rows(wl: Workload, n: int, seed: int = 0) -> np.ndarray:
     rest = rng.choice(total, size=n, replace=False)
     rows = list(fixed) + [int(x) for x in rest if int(x) not in fixed]
     return np.sort(np.asarray(rows[:n], dtype=np.int64))
+
+
+# ---------------------------------------------------------------------------------------------
+# Prompt groups: the paper's GRPO setting scores N sampled responses per prompt and computes the
+# prompt prefix once per group (Section 4.1 lists N = 8 and enables prefix sharing in every system).
+# ---------------------------------------------------------------------------------------------
+@dataclass
+class GroupWorkload:
+    """B prompts with `group` responses each.
+
+    `prompts` is a Workload whose sequences are the B prompts alone (response length 0): its
+    prefix-packed tensors feed the one prefix pass per prompt.  `members` is a Workload of the
+    B * group whole sequences (prompt tokens repeated bit for bit in every member, then that
+    member's response): the oracle scores those one by one, and their suffix-packed tensors feed
+    the suffix pass.  `member_table` is the block table of the suffix pass: member m of prompt b
+    uses row b of the prompts' table, so all members of a group read the same cache blocks.
+    """
+
+    group: int
+    prompts: Workload
+    members: Workload
+    member_table: np.ndarray
+
+
+def make_group_workload(cfg: Config, group: int, seed: int = 0) -> GroupWorkload:
+    """cfg.batch prompts drawn as in make_workload; each gets `group` responses of its own length."""
+    lrng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, _TENSOR_IDS["lengths"], 1])))
+    p = draw_lengths(cfg.prompt, cfg.batch, lrng)
+    prompt_cfg = cfg.scaled(name=cfg.name + "-prompts", prompt=("list", [int(x) for x in p]),
+                            response=("list", [0] * cfg.batch))
+    prompts = make_workload(prompt_cfg, seed=seed)
+    n_members = cfg.batch * group
+    r = draw_lengths(cfg.response, n_members, lrng)
+    member_cfg = cfg.scaled(name=cfg.name + f"-x{group}", batch=n_members, prompt=("list", [int(x) for x in np.repeat(p, group)]),
+                            response=("list", [int(x) for x in r]))
+    members = make_workload(member_cfg, seed=seed + 1000003)
+    # overwrite every member's prompt tokens with its prompt's tensors so the prefix really is shared
+    for m in range(n_members):
+        b = m // group
+        src = slice(int(prompts.cu_full[b]), int(prompts.cu_full[b + 1]))
+        dst = slice(int(members.cu_full[m]), int(members.cu_full[m]) + int(p[b]))
+        for name in ("q", "k", "v", "hidden", "ids"):
+            getattr(members, name)[dst] = getattr(prompts, name)[src]
+    members.w = prompts.w
+    member_table = np.repeat(prompts.block_table, group, axis=0)
+    members.block_table = member_table
+    members.num_blocks = prompts.num_blocks
+    return GroupWorkload(group, prompts, members, member_table)
