@@ -403,7 +403,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))
-    ap.add_argument("--cpu-tokens", type=int, default=48, help="tokens the oracle scores for cpu_baseline")
+    ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--group", type=int, default=0, help="score prompt groups of this size (prefix once per prompt)")

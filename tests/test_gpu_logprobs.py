@@ -110,3 +110,14 @@ def test_c2_full_size_sampled_rows(cuda_device):
     assert np.abs(lp - ref_lp).max() <= TIGHT
     assert np.abs(lse - ref_lse).max() <= TIGHT
     assert abs(ref_lp.mean() + (np.log(152064) + 0.5 * 3584 * 0.02 ** 2)) < 0.6
+
+
+@pytest.mark.parametrize("name", ["C3", "C4", "C5"])
+def test_other_full_size_configs_sampled_rows(cuda_device, name):
+    """The remaining BASELINE configs at full size (32B shape: hidden 5120; C3 has ~226 k rows, C5
+    ~135 k), 24 sampled rows each against the oracle."""
+    wl = wk.make_workload(wk.CONFIGS[name], seed=0, attn=False)
+    rows = wk.sample_logprob_rows(wl, 24, seed=3)
+    lp, lse, ref_lp, ref_lse = _run(wl, cuda_device, rows)
+    assert np.abs(lp - ref_lp).max() <= TIGHT
+    assert np.abs(lse - ref_lse).max() <= TIGHT
