@@ -50,6 +50,8 @@ def _load():
                                              i32, dbl, vp, i64, vp, vp]
         lib.rpx_oracle_logprob_rows.restype = ctypes.c_int
         lib.rpx_oracle_logprob_rows.argtypes = [vp, i64, vp, ctypes.c_int, vp, vp, i64, i32, i32, vp, vp]
+        lib.rpx_oracle_entropy_rows.restype = ctypes.c_int
+        lib.rpx_oracle_entropy_rows.argtypes = [vp, i64, vp, ctypes.c_int, vp, i64, i32, i32, vp]
         lib.rpx_oracle_slot.restype = i64
         lib.rpx_oracle_slot.argtypes = [vp, i32, i32, i32, i32]
         lib.rpx_oracle_cache_image.restype = ctypes.c_int
@@ -142,6 +144,23 @@ def logprob_rows(hidden, w, target_ids, rows=None):
     if rc != 0:
         raise MemoryError(f"rpx_oracle_logprob_rows failed with {rc}")
     return lp, lse
+
+
+def entropy_rows(hidden, w, rows=None):
+    """Entropy (nats) of softmax(hidden[n] . w^T) per row, from the definition -sum p ln p in fp64."""
+    lib = _load()
+    code = _dtype_code(hidden)
+    assert _dtype_code(w) == code and hidden.ndim == 2 and w.ndim == 2 and hidden.shape[1] == w.shape[1]
+    assert hidden.strides[1] == hidden.itemsize and w.flags.c_contiguous
+    if rows is None:
+        rows = np.arange(hidden.shape[0], dtype=np.int64)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    ent = np.empty((rows.shape[0],), dtype=np.float64)
+    rc = lib.rpx_oracle_entropy_rows(_ptr(hidden), hidden.strides[0] // hidden.itemsize, _ptr(w), code, _ptr(rows),
+                                     rows.shape[0], hidden.shape[1], w.shape[0], _ptr(ent))
+    if rc != 0:
+        raise MemoryError(f"rpx_oracle_entropy_rows failed with {rc}")
+    return ent
 
 
 def slot(block_table, s: int, t: int, block_size: int = 16) -> int:

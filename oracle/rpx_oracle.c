@@ -17,6 +17,7 @@
  *   log-prob    for row n:  z_v = sum_c hidden[n,c] * W[v,c]           v = 0..V-1
  *                   logprob[n] = z_target - (max_v z_v + ln sum_v exp(z_v - max_v z_v))
  *   slot map    slot(s,t) = block_table[s][t / block_size] * block_size + t % block_size
+ *   entropy     (extension) H[n] = - sum_v p_v ln p_v with p = softmax(z[n,:])
  *
  * Every input element is promoted to double first; sums run in index order with no blocking.
  * Pins (tests/test_oracle_pins.py): brute force on tiny inputs in extended precision with a
@@ -155,6 +156,48 @@ int rpx_oracle_logprob_rows(const void* hidden, int64_t hidden_row_stride, const
         const int32_t t = target_ids[rows[r]];
         logprob[r] = (t >= 0 && t < vocab) ? zr[t] - ls : NAN;
         if (lse) lse[r] = ls;
+    }
+    free(z);
+    return 0;
+}
+
+/*
+ * Entropy of the next-token distribution for a list of rows (an extension beyond the paper, which
+ * only needs log-probs): with p_v = exp(z_v - lse),  H[n] = - sum_v p_v * ln p_v, written out as
+ * that definition in double (terms with p_v == 0 contribute 0).
+ */
+int rpx_oracle_entropy_rows(const void* hidden, int64_t hidden_row_stride, const void* w, int dtype,
+                            const int64_t* rows, int64_t n_rows, int32_t hidden_dim, int32_t vocab,
+                            double* entropy) {
+    double* z = (double*)malloc(sizeof(double) * (size_t)n_rows * (size_t)vocab);
+    if (!z) return -2;
+#pragma omp parallel for schedule(static)
+    for (int32_t vv = 0; vv < vocab; ++vv) {
+        const int64_t woff = (int64_t)vv * hidden_dim;
+        for (int64_t r = 0; r < n_rows; ++r) {
+            const int64_t hoff = rows[r] * hidden_row_stride;
+            double dot = 0.0;
+            for (int c = 0; c < hidden_dim; ++c)
+                dot += load_elem(hidden, dtype, hoff + c) * load_elem(w, dtype, woff + c);
+            z[r * (int64_t)vocab + vv] = dot;
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const double* zr = z + r * (int64_t)vocab;
+        double m = -INFINITY;
+        for (int32_t vv = 0; vv < vocab; ++vv)
+            if (zr[vv] > m) m = zr[vv];
+        double l = 0.0;
+        for (int32_t vv = 0; vv < vocab; ++vv) l += exp(zr[vv] - m);
+        const double ls = m + log(l);
+        double h = 0.0;
+        for (int32_t vv = 0; vv < vocab; ++vv) {
+            const double lp = zr[vv] - ls;
+            const double pv = exp(lp);
+            if (pv > 0.0) h -= pv * lp;
+        }
+        entropy[r] = h;
     }
     free(z);
     return 0;

@@ -347,3 +347,36 @@ def test_length_recipes():
         assert lo_share <= share <= hi_share, (name, share)
     p = wk.draw_lengths(("lognormal", 6000, 0.5, 1024, 16384), 2000, np.random.default_rng(0))
     assert p.min() >= 1024 and p.max() <= 16384 and abs(np.median(p) - 6000) < 300
+
+
+# ---------------------------------------------------------------- entropy (extension) pins
+def test_entropy_closed_forms_bounds_and_torch():
+    vocab, h = 64, 12
+    hid = _rand((5, h), 200)
+    # uniform distribution: ln V
+    ent = oracle.entropy_rows(hid, np.zeros((vocab, h), np.float32))
+    assert np.abs(ent - math.log(vocab)).max() < 1e-13
+    # two classes with logits (a, 0): the binary entropy of sigmoid(a), typed out independently
+    w2 = np.zeros((2, h), np.float32)
+    w2[0, 0] = 1.0
+    hid2 = np.zeros((4, h), np.float32)
+    hid2[:, 0] = [0.0, 1.5, -3.0, 30.0]
+    ent2 = oracle.entropy_rows(hid2, w2)
+    for a, got in zip([0.0, 1.5, -3.0, 30.0], ent2):
+        p1 = 1.0 / (1.0 + math.exp(-a))
+        ref = -(p1 * math.log(p1) + (1 - p1) * math.log1p(-p1)) if p1 < 1.0 else 0.0
+        assert abs(got - ref) < 1e-12
+    # bounds, and the library routine in fp64
+    w = _rand((vocab, h), 201, 0.7)
+    ent3 = oracle.entropy_rows(hid, w)
+    assert (ent3 > 0).all() and (ent3 < math.log(vocab)).all()
+    logits = torch.from_numpy(hid).double() @ torch.from_numpy(w).double().T
+    ref = torch.distributions.Categorical(logits=logits).entropy().numpy()
+    np.testing.assert_allclose(ent3, ref, rtol=0, atol=1e-12)
+    # consistency with the log-prob oracle: H = lse - E_p[z]
+    _, lse = oracle.logprob_rows(hid, w, np.zeros(5, np.int32))
+    z = logits.numpy()
+    pr = np.exp(z - lse[:, None])
+    np.testing.assert_allclose(ent3, lse - (pr * z).sum(axis=1), rtol=0, atol=1e-12)
+    sub = oracle.entropy_rows(hid, w, rows=np.array([4, 1], np.int64))
+    assert (sub == ent3[[4, 1]]).all()
