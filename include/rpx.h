@@ -145,6 +145,19 @@ RPX_API rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_s
                                 void* cuda_stream);
 
 /*
+ * rpx_token_logprobs with one more output from the same pass (an extension; the paper only needs
+ * the log-probs): entropy[n] = - sum_v p_v ln p_v of the next-token distribution p = softmax(z[n,:]),
+ * float32 [n_tokens], nullable.  It costs one more multiply-add per logit in the epilogue and no
+ * extra memory traffic; every other argument, the workspace size and the error behaviour are those
+ * of rpx_token_logprobs (which is this call with entropy == NULL).
+ */
+RPX_API rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
+                                                int32_t vocab, rpx_dtype_t dtype, float* logprobs, float* lse,
+                                                float* entropy, void* workspace, size_t workspace_bytes,
+                                                int32_t* device_status, void* cuda_stream);
+
+/*
  * Allocation-free variant of rpx_token_logprobs (the paper has no counterpart: this entry point
  * exists for deployment, not for the method).  It is meant for callers that cannot give the
  * library a workspace because they cannot allocate one: a scoring hook that runs inside an

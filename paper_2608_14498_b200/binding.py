@@ -22,6 +22,7 @@ EXPORTS = (
     "rpx_prefix_attn",
     "rpx_suffix_attn",
     "rpx_token_logprobs",
+    "rpx_token_logprobs_entropy",
     "rpx_token_logprobs_static",
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
@@ -83,6 +84,8 @@ def load_library():
                                     i32, ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs.restype = i32
     lib.rpx_token_logprobs.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_entropy.restype = i32
+    lib.rpx_token_logprobs_entropy.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs_static.restype = i32
     lib.rpx_token_logprobs_static.argtypes = [vp, i64, vp, vp, i64, i32, i32, vp, vp, vp, vp]
     lib.rpx_prefix_attn_workspace_bytes.restype = sz
@@ -243,8 +246,11 @@ def suffix_attn(q, k, v, cu_seqlens_suffix, prefix_lens, max_suffix_len: int, ma
 
 
 def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_lse: bool = False, workspace=None,
-                   device_status=None, stream=None):
-    """rpx_token_logprobs: log p(target) per row from hidden [N, H] and W [V, H]; logits never stored."""
+                   device_status=None, stream=None, entropy=None):
+    """rpx_token_logprobs: log p(target) per row from hidden [N, H] and W [V, H]; logits never stored.
+
+    ``entropy`` (float32 [N], optional) additionally receives the entropy of each row's next-token
+    distribution from the same pass (rpx_token_logprobs_entropy)."""
     torch = _torch()
     lib = load_library()
     code = _dtype_code(hidden)
@@ -260,9 +266,14 @@ def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_
         lse = torch.empty((n,), dtype=torch.float32, device=hidden.device)
     ws = _workspace(int(lib.rpx_token_logprobs_workspace_bytes(n, hdim, vocab, code)), hidden.device, workspace)
     row_stride = hidden.stride(0) if n > 1 else hdim
-    rc = lib.rpx_token_logprobs(_ptr(hidden), row_stride, _ptr(w_vocab), _ptr(target_ids), n, hdim, vocab, code,
-                                _ptr(logprobs), _ptr(lse), _ptr(ws), ws.numel() * ws.element_size(),
-                                _ptr(device_status), _stream_ptr(stream))
+    if entropy is None:
+        rc = lib.rpx_token_logprobs(_ptr(hidden), row_stride, _ptr(w_vocab), _ptr(target_ids), n, hdim, vocab, code,
+                                    _ptr(logprobs), _ptr(lse), _ptr(ws), ws.numel() * ws.element_size(),
+                                    _ptr(device_status), _stream_ptr(stream))
+    else:
+        rc = lib.rpx_token_logprobs_entropy(_ptr(hidden), row_stride, _ptr(w_vocab), _ptr(target_ids), n, hdim, vocab,
+                                            code, _ptr(logprobs), _ptr(lse), _ptr(entropy), _ptr(ws),
+                                            ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
         raise RpxError(rc, "rpx_token_logprobs")
     return (logprobs, lse) if return_lse else logprobs

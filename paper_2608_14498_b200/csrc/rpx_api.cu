@@ -149,10 +149,10 @@ size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, 
     return bytes;
 }
 
-rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
-                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
-                                rpx_dtype_t dtype, float* logprobs, float* lse, void* workspace, size_t workspace_bytes,
-                                int32_t* device_status, void* cuda_stream) {
+rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                        const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                        rpx_dtype_t dtype, float* logprobs, float* lse, float* entropy, void* workspace,
+                                        size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
     if (dtype != RPX_BF16 && dtype != RPX_F32) return RPX_ERR_DTYPE;
     if (n_tokens < 0 || n_tokens >= INT32_MAX || hidden_dim <= 0 || vocab <= 0) return RPX_ERR_SHAPE;
     if (hidden_dim % 8 != 0) return RPX_ERR_SHAPE;
@@ -191,9 +191,18 @@ rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, c
     a.vocab = vocab;
     a.logprobs = logprobs;
     a.lse = lse;
+    a.entropy = entropy;
     a.device_status = device_status;
     a.stream = stream;
     return launch_token_logprobs(a);
+}
+
+rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                rpx_dtype_t dtype, float* logprobs, float* lse, void* workspace, size_t workspace_bytes,
+                                int32_t* device_status, void* cuda_stream) {
+    return rpx_token_logprobs_entropy(hidden, hidden_row_stride, w_vocab, target_ids, n_tokens, hidden_dim, vocab, dtype,
+                                      logprobs, lse, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
 }
 
 rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* device_status, void* cuda_stream) {

@@ -52,6 +52,7 @@ struct LogprobArgs {
     int32_t hidden_dim, vocab;
     float* logprobs;
     float* lse;
+    float* entropy;       // nullable
     void* partials;       // float4 [logprob_num_chunks(vocab, tiles_per_chunk)][n_tokens]
     int32_t tiles_per_chunk;  // vocabulary tiles (256 columns) one work item sweeps
     int32_t* device_status;

@@ -57,7 +57,8 @@ struct Params {
     int32_t group_width;   // vocab chunks in flight side by side
     int32_t total_items;
     const int32_t* target_ids;
-    float4* partials;      // [n_chunks][n_rows]: (max in log2 units, sum of 2^(x-max), target logit, 0)
+    float4* partials;      // [n_chunks][n_rows]: (max in log2 units, sum of 2^(x-max), target logit,
+                           //                      sum of 2^(x-max) * z  -- for the entropy)
     int32_t* status;
 };
 
@@ -196,7 +197,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const int64_t row = static_cast<int64_t>(item.m_tile) * kBM + row_in_tile;
             const bool valid = row < p.n_rows;
             const int32_t target = valid ? __ldg(p.target_ids + row) : -1;
-            float run_max = -CUDART_INF_F, run_sum = 0.f, target_logit = 0.f;
+            float run_max = -CUDART_INF_F, run_sum = 0.f, target_logit = 0.f, run_wsum = 0.f;
             for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
                 const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
                 if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) {
@@ -234,11 +235,18 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                             if (tl == static_cast<uint32_t>(i)) target_logit = __uint_as_float(r[i]);
                     }
                     const float new_max = fmaxf(run_max, cmax);
-                    run_sum *= fast_exp2(run_max - new_max);
-                    float part = 0.f;
+                    const float shrink = fast_exp2(run_max - new_max);
+                    run_sum *= shrink;
+                    run_wsum *= shrink;
+                    float part = 0.f, wpart = 0.f;  // sum of weights, and of weight * logit (entropy)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) part += fast_exp2(x[i] - new_max);
+                    for (int i = 0; i < 32; ++i) {
+                        const float e = fast_exp2(x[i] - new_max);  // 0 for masked columns (x = -inf)
+                        part += e;
+                        wpart = fmaf(e, __uint_as_float(r[i]), wpart);
+                    }
                     run_sum += part;
+                    run_wsum += wpart;
                     run_max = new_max;
                 }
                 tc_fence_before_sync();
@@ -246,7 +254,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             }
             if (ok && valid)
                 p.partials[static_cast<int64_t>(item.chunk) * p.n_rows + row] =
-                    make_float4(run_max, run_sum, target_logit, 0.f);
+                    make_float4(run_max, run_sum, target_logit, run_wsum);
         }
     }
 
@@ -261,15 +269,18 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
 __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int32_t n_chunks, int64_t n_rows,
                                        const int32_t* __restrict__ target_ids, int32_t vocab,
-                                       float* __restrict__ logprobs, float* __restrict__ lse, int32_t* status) {
+                                       float* __restrict__ logprobs, float* __restrict__ lse,
+                                       float* __restrict__ entropy, int32_t* status) {
     const int64_t row = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (row >= n_rows) return;
     float gmax = -CUDART_INF_F;
     for (int32_t c = 0; c < n_chunks; ++c) gmax = fmaxf(gmax, partials[static_cast<int64_t>(c) * n_rows + row].x);
-    float sum = 0.f, zt = 0.f;
+    float sum = 0.f, zt = 0.f, wsum = 0.f;
     for (int32_t c = 0; c < n_chunks; ++c) {
         const float4 v = partials[static_cast<int64_t>(c) * n_rows + row];
-        sum += v.y * exp2f(v.x - gmax);
+        const float f = exp2f(v.x - gmax);
+        sum += v.y * f;
+        wsum += v.w * f;
         zt += v.z;
     }
     const float l = (gmax + log2f(sum)) * kLn2;
@@ -283,6 +294,8 @@ __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int3
     }
     logprobs[row] = lp;
     if (lse != nullptr) lse[row] = l;
+    // H = -sum_v p_v ln p_v = lse - E_p[z]
+    if (entropy != nullptr) entropy[row] = l - wsum / sum;
 }
 
 }  // namespace
@@ -342,7 +355,7 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     const int cthreads = 256;
     const unsigned cblocks = static_cast<unsigned>((a.n_tokens + cthreads - 1) / cthreads);
     lm_head_combine_kernel<<<cblocks, cthreads, 0, a.stream>>>(p.partials, p.n_chunks, a.n_tokens, a.target_ids,
-                                                               a.vocab, a.logprobs, a.lse, a.device_status);
+                                                               a.vocab, a.logprobs, a.lse, a.entropy, a.device_status);
     return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
 }
 
@@ -411,6 +424,7 @@ extern "C" RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, in
     a.vocab = vocab;
     a.logprobs = logprobs;
     a.lse = lse;
+    a.entropy = nullptr;
     a.partials = scratch;
     a.tiles_per_chunk = kTilesPerChunkLarge;  // the documented size limit assumes 16-tile chunks
     a.device_status = device_status;

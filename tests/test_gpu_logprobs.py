@@ -121,3 +121,26 @@ def test_other_full_size_configs_sampled_rows(cuda_device, name):
     lp, lse, ref_lp, ref_lse = _run(wl, cuda_device, rows)
     assert np.abs(lp - ref_lp).max() <= TIGHT
     assert np.abs(lse - ref_lse).max() <= TIGHT
+
+
+@pytest.mark.parametrize("n_tokens,hidden,vocab,scale", [(300, 200, 1000, 1.0), (257, 512, 5000, 1.0), (200, 256, 2048, 40.0)])
+def test_entropy_from_the_same_pass(cuda_device, n_tokens, hidden, vocab, scale):
+    """rpx_token_logprobs_entropy: H = -sum p ln p per row against the oracle's definition, on ragged
+    shapes, several chunks, and peaked distributions (logits of a few hundred, entropy near 0)."""
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, hidden, vocab, ("fixed", n_tokens), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=8, attn=False)
+    if scale != 1.0:
+        w = wk.bf16_bits_to_f32(wl.w).reshape(wl.w.shape) * scale
+        wl.w = wk.f32_to_bf16_bits(w).reshape(w.shape)
+    h, w, ids = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    ent = torch.full((n_tokens,), float("nan"), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    lp = rpx.token_logprobs(h, w, ids, entropy=ent, device_status=status)
+    lp_plain = rpx.token_logprobs(h, w, ids)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(lp, lp_plain)
+    ref = oracle.entropy_rows(wl.hidden, wl.w)
+    got = ent.double().cpu().numpy()
+    assert np.isfinite(got).all() and (got > -1e-3).all() and (got < np.log(vocab) + 1e-3).all()
+    assert np.abs(got - ref).max() <= TIGHT + 1e-5 * np.abs(ref).max() * (scale > 1)
