@@ -158,6 +158,27 @@ RPX_API rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidd
                                                 int32_t* device_status, void* cuda_stream);
 
 /*
+ * Vocabulary-parallel LM head (an extension; it is how a tensor-parallel reference model, such as
+ * the paper's TP=8 one, lays out its LM head).  Each rank holds the rows vocab_begin ..
+ * vocab_begin + vocab_local - 1 of W_vocab and calls rpx_token_logprobs_shard on the full hidden
+ * rows; the call leaves one 16-byte record per row in shard_stats (float [n_tokens][4], 16-byte
+ * aligned): (running max in log2 units, sum of 2^(x - max), target logit if the target lies in
+ * this shard else 0, sum of 2^(x - max) * logit).  The ranks exchange their records (one
+ * all-gather of 16 bytes per row and rank) and every rank calls rpx_token_logprobs_merge on the
+ * gathered array float [n_shards][n_tokens][4]; the result equals rpx_token_logprobs(_entropy) on
+ * the whole vocabulary up to fp32 summation order.  target_ids hold GLOBAL vocabulary ids in both
+ * calls; workspace as rpx_token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab_local, dtype).
+ */
+RPX_API rpx_status_t rpx_token_logprobs_shard(const void* hidden, int64_t hidden_row_stride, const void* w_shard,
+                                              const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
+                                              int32_t vocab_local, int32_t vocab_begin, rpx_dtype_t dtype,
+                                              float* shard_stats, void* workspace, size_t workspace_bytes,
+                                              int32_t* device_status, void* cuda_stream);
+RPX_API rpx_status_t rpx_token_logprobs_merge(const float* shard_stats, int32_t n_shards, const int32_t* target_ids,
+                                              int64_t n_tokens, int32_t vocab_total, float* logprobs, float* lse,
+                                              float* entropy, int32_t* device_status, void* cuda_stream);
+
+/*
  * Allocation-free variant of rpx_token_logprobs (the paper has no counterpart: this entry point
  * exists for deployment, not for the method).  It is meant for callers that cannot give the
  * library a workspace because they cannot allocate one: a scoring hook that runs inside an

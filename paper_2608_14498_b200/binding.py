@@ -23,6 +23,8 @@ EXPORTS = (
     "rpx_suffix_attn",
     "rpx_token_logprobs",
     "rpx_token_logprobs_entropy",
+    "rpx_token_logprobs_shard",
+    "rpx_token_logprobs_merge",
     "rpx_token_logprobs_static",
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
@@ -86,6 +88,10 @@ def load_library():
     lib.rpx_token_logprobs.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs_entropy.restype = i32
     lib.rpx_token_logprobs_entropy.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_shard.restype = i32
+    lib.rpx_token_logprobs_shard.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_merge.restype = i32
+    lib.rpx_token_logprobs_merge.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp, vp]
     lib.rpx_token_logprobs_static.restype = i32
     lib.rpx_token_logprobs_static.argtypes = [vp, i64, vp, vp, i64, i32, i32, vp, vp, vp, vp]
     lib.rpx_prefix_attn_workspace_bytes.restype = sz
@@ -302,3 +308,47 @@ def token_logprobs_static(hidden, w_vocab, target_ids, logprobs, lse=None, devic
     if rc != 0:
         raise RpxError(rc, "rpx_token_logprobs_static")
     return logprobs
+
+
+def token_logprobs_shard(hidden, w_shard, target_ids, vocab_begin: int, shard_stats=None, workspace=None,
+                         device_status=None, stream=None):
+    """rpx_token_logprobs_shard: this rank's share of a vocabulary-parallel LM head.
+
+    w_shard holds rows vocab_begin .. vocab_begin + V_local - 1 of W_vocab; target_ids are global ids.
+    Returns shard_stats float32 [N, 4] to be gathered over ranks and passed to token_logprobs_merge."""
+    torch = _torch()
+    lib = load_library()
+    code = _dtype_code(hidden)
+    if _dtype_code(w_shard) != code:
+        raise TypeError("hidden and w_shard must share an element type")
+    if hidden.dim() != 2 or hidden.stride(1) != 1 or not w_shard.is_contiguous():
+        raise ValueError("hidden must be [N, H] with contiguous rows and w_shard contiguous [V_local, H]")
+    n, hdim = hidden.shape
+    v_local = w_shard.shape[0]
+    if shard_stats is None:
+        shard_stats = torch.empty((n, 4), dtype=torch.float32, device=hidden.device)
+    ws = _workspace(int(lib.rpx_token_logprobs_workspace_bytes(n, hdim, v_local, code)), hidden.device, workspace)
+    rc = lib.rpx_token_logprobs_shard(_ptr(hidden), hidden.stride(0) if n > 1 else hdim, _ptr(w_shard), _ptr(target_ids), n,
+                                      hdim, v_local, int(vocab_begin), code, _ptr(shard_stats), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_token_logprobs_shard")
+    return shard_stats
+
+
+def token_logprobs_merge(all_stats, target_ids, vocab_total: int, logprobs=None, return_lse: bool = False, entropy=None,
+                         device_status=None, stream=None):
+    """rpx_token_logprobs_merge: final log-probs from the gathered shard records float32 [R, N, 4]."""
+    torch = _torch()
+    lib = load_library()
+    if all_stats.dim() != 3 or all_stats.shape[2] != 4 or all_stats.dtype != torch.float32 or not all_stats.is_contiguous():
+        raise ValueError("all_stats must be a contiguous float32 [shards, N, 4] tensor")
+    r, n, _ = all_stats.shape
+    if logprobs is None:
+        logprobs = torch.empty((n,), dtype=torch.float32, device=all_stats.device)
+    lse = torch.empty((n,), dtype=torch.float32, device=all_stats.device) if return_lse else None
+    rc = lib.rpx_token_logprobs_merge(_ptr(all_stats), r, _ptr(target_ids), n, int(vocab_total), _ptr(logprobs), _ptr(lse),
+                                      _ptr(entropy), _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_token_logprobs_merge")
+    return (logprobs, lse) if return_lse else logprobs

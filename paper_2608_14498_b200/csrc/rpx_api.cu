@@ -149,18 +149,27 @@ size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, 
     return bytes;
 }
 
-rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
-                                        const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
-                                        rpx_dtype_t dtype, float* logprobs, float* lse, float* entropy, void* workspace,
-                                        size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Shared body of the LM-head entry points.  shard_stats != NULL selects the vocabulary-shard form
+// (W holds columns vocab_begin .. vocab_begin + vocab - 1; the merged record per row is the output).
+rpx_status_t run_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                int32_t vocab_begin, rpx_dtype_t dtype, float* logprobs, float* lse, float* entropy,
+                                float* shard_stats, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                void* cuda_stream) {
     if (dtype != RPX_BF16 && dtype != RPX_F32) return RPX_ERR_DTYPE;
     if (n_tokens < 0 || n_tokens >= INT32_MAX || hidden_dim <= 0 || vocab <= 0) return RPX_ERR_SHAPE;
     if (hidden_dim % 8 != 0) return RPX_ERR_SHAPE;
     if (n_tokens == 0) return RPX_OK;
-    if (hidden == nullptr || w_vocab == nullptr || target_ids == nullptr || logprobs == nullptr) return RPX_ERR_NULL;
+    if (hidden == nullptr || w_vocab == nullptr || target_ids == nullptr) return RPX_ERR_NULL;
+    if (logprobs == nullptr && shard_stats == nullptr) return RPX_ERR_NULL;
+    if (vocab_begin < 0) return RPX_ERR_SHAPE;
     if (hidden_row_stride < hidden_dim) return RPX_ERR_SHAPE;
     if (hidden_row_stride % 8 != 0) return RPX_ERR_ALIGN;
-    if (!aligned16(hidden) || !aligned16(w_vocab)) return RPX_ERR_ALIGN;
+    if (!aligned16(hidden) || !aligned16(w_vocab) || !aligned16(shard_stats)) return RPX_ERR_ALIGN;
     const size_t need = rpx_token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype);
     if (workspace == nullptr || workspace_bytes < need) return RPX_ERR_WORKSPACE;
     if (!aligned16(workspace)) return RPX_ERR_ALIGN;
@@ -192,9 +201,46 @@ rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidden_row_s
     a.logprobs = logprobs;
     a.lse = lse;
     a.entropy = entropy;
+    a.shard_stats = shard_stats;
+    a.target_offset = vocab_begin;
     a.device_status = device_status;
     a.stream = stream;
     return launch_token_logprobs(a);
+}
+
+}  // namespace
+
+extern "C" {
+
+rpx_status_t rpx_token_logprobs_entropy(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                        const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                        rpx_dtype_t dtype, float* logprobs, float* lse, float* entropy, void* workspace,
+                                        size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    return run_token_logprobs(hidden, hidden_row_stride, w_vocab, target_ids, n_tokens, hidden_dim, vocab, 0, dtype,
+                              logprobs, lse, entropy, nullptr, workspace, workspace_bytes, device_status, cuda_stream);
+}
+
+rpx_status_t rpx_token_logprobs_shard(const void* hidden, int64_t hidden_row_stride, const void* w_shard,
+                                      const int32_t* target_ids, int64_t n_tokens, int32_t hidden_dim,
+                                      int32_t vocab_local, int32_t vocab_begin, rpx_dtype_t dtype, float* shard_stats,
+                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                      void* cuda_stream) {
+    if (n_tokens > 0 && shard_stats == nullptr) return RPX_ERR_NULL;
+    return run_token_logprobs(hidden, hidden_row_stride, w_shard, target_ids, n_tokens, hidden_dim, vocab_local,
+                              vocab_begin, dtype, nullptr, nullptr, nullptr, shard_stats, workspace, workspace_bytes,
+                              device_status, cuda_stream);
+}
+
+rpx_status_t rpx_token_logprobs_merge(const float* shard_stats, int32_t n_shards, const int32_t* target_ids,
+                                      int64_t n_tokens, int32_t vocab_total, float* logprobs, float* lse, float* entropy,
+                                      int32_t* device_status, void* cuda_stream) {
+    if (n_shards <= 0 || n_tokens < 0 || n_tokens >= INT32_MAX || vocab_total <= 0) return RPX_ERR_SHAPE;
+    if (n_tokens == 0) return RPX_OK;
+    if (shard_stats == nullptr || target_ids == nullptr || logprobs == nullptr) return RPX_ERR_NULL;
+    if (!aligned16(shard_stats)) return RPX_ERR_ALIGN;
+    if (rpx_status_t rc = check_arch()) return rc;
+    return launch_logprob_merge(shard_stats, n_shards, target_ids, n_tokens, vocab_total, logprobs, lse, entropy,
+                                device_status, static_cast<cudaStream_t>(cuda_stream));
 }
 
 rpx_status_t rpx_token_logprobs(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,

@@ -53,6 +53,8 @@ struct LogprobArgs {
     float* logprobs;
     float* lse;
     float* entropy;       // nullable
+    void* shard_stats;    // nullable float4 [n_tokens]: emit the merged record instead of final outputs
+    int32_t target_offset;  // first vocabulary column of `w` (vocabulary-parallel shards), else 0
     void* partials;       // float4 [logprob_num_chunks(vocab, tiles_per_chunk)][n_tokens]
     int32_t tiles_per_chunk;  // vocabulary tiles (256 columns) one work item sweeps
     int32_t* device_status;
@@ -61,6 +63,9 @@ struct LogprobArgs {
 int32_t logprob_tiles_per_chunk(int64_t n_tokens);  // the default policy
 int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk);
 rpx_status_t launch_token_logprobs(const LogprobArgs& a);
+rpx_status_t launch_logprob_merge(const void* shard_stats, int32_t n_shards, const int32_t* target_ids, int64_t n_tokens,
+                                  int32_t vocab_total, float* logprobs, float* lse, float* entropy, int32_t* status,
+                                  cudaStream_t stream);
 
 rpx_status_t launch_bounded_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t stream);
 

@@ -57,6 +57,7 @@ struct Params {
     int32_t group_width;   // vocab chunks in flight side by side
     int32_t total_items;
     const int32_t* target_ids;
+    int32_t target_offset; // first vocabulary column of this W (0 unless W is one shard of the vocabulary)
     float4* partials;      // [n_chunks][n_rows]: (max in log2 units, sum of 2^(x-max), target logit,
                            //                      sum of 2^(x-max) * z  -- for the entropy)
     int32_t* status;
@@ -196,7 +197,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const Item item = decode_item(p, idx);
             const int64_t row = static_cast<int64_t>(item.m_tile) * kBM + row_in_tile;
             const bool valid = row < p.n_rows;
-            const int32_t target = valid ? __ldg(p.target_ids + row) : -1;
+            const int32_t target = valid ? __ldg(p.target_ids + row) - p.target_offset : -1;
             float run_max = -CUDART_INF_F, run_sum = 0.f, target_logit = 0.f, run_wsum = 0.f;
             for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
                 const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
@@ -270,7 +271,7 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int32_t n_chunks, int64_t n_rows,
                                        const int32_t* __restrict__ target_ids, int32_t vocab,
                                        float* __restrict__ logprobs, float* __restrict__ lse,
-                                       float* __restrict__ entropy, int32_t* status) {
+                                       float* __restrict__ entropy, float4* __restrict__ stats_out, int32_t* status) {
     const int64_t row = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x;
     if (row >= n_rows) return;
     float gmax = -CUDART_INF_F;
@@ -282,6 +283,10 @@ __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int3
         sum += v.y * f;
         wsum += v.w * f;
         zt += v.z;
+    }
+    if (stats_out != nullptr) {  // one vocabulary shard: hand the merged record on, another launch finishes
+        stats_out[row] = make_float4(gmax, sum, zt, wsum);
+        return;
     }
     const float l = (gmax + log2f(sum)) * kLn2;
     const int32_t t = target_ids[row];
@@ -340,22 +345,31 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     const int grid = static_cast<int>(total < sms ? total : sms);
     p.group_width = (grid % 4 == 0) ? 4 : (grid % 2 == 0 ? 2 : 1);
     p.target_ids = a.target_ids;
+    p.target_offset = a.target_offset;
     p.partials = static_cast<float4*>(a.partials);
     p.status = a.device_status;
 
-    static bool attr_set = false;  // idempotent; a race only repeats the call
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(lm_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kSmemBytes)) != cudaSuccess)
-            return RPX_ERR_CUDA;
-        attr_set = true;
-    }
+    if (cudaFuncSetAttribute(lm_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kSmemBytes)) != cudaSuccess)  // per device, cheap: set every time
+        return RPX_ERR_CUDA;
     lm_head_partial_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w, p);
     if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
     const int cthreads = 256;
     const unsigned cblocks = static_cast<unsigned>((a.n_tokens + cthreads - 1) / cthreads);
     lm_head_combine_kernel<<<cblocks, cthreads, 0, a.stream>>>(p.partials, p.n_chunks, a.n_tokens, a.target_ids,
-                                                               a.vocab, a.logprobs, a.lse, a.entropy, a.device_status);
+                                                               a.vocab, a.logprobs, a.lse, a.entropy,
+                                                               static_cast<float4*>(a.shard_stats), a.device_status);
+    return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
+}
+
+rpx_status_t launch_logprob_merge(const void* shard_stats, int32_t n_shards, const int32_t* target_ids, int64_t n_tokens,
+                                  int32_t vocab_total, float* logprobs, float* lse, float* entropy, int32_t* status,
+                                  cudaStream_t stream) {
+    if (n_tokens == 0) return RPX_OK;
+    const int cthreads = 256;
+    const unsigned cblocks = static_cast<unsigned>((n_tokens + cthreads - 1) / cthreads);
+    lm_head_combine_kernel<<<cblocks, cthreads, 0, stream>>>(static_cast<const float4*>(shard_stats), n_shards, n_tokens,
+                                                             target_ids, vocab_total, logprobs, lse, entropy, nullptr, status);
     return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
 }
 
@@ -425,6 +439,8 @@ extern "C" RPX_API rpx_status_t rpx_token_logprobs_static(const void* hidden, in
     a.logprobs = logprobs;
     a.lse = lse;
     a.entropy = nullptr;
+    a.shard_stats = nullptr;
+    a.target_offset = 0;
     a.partials = scratch;
     a.tiles_per_chunk = kTilesPerChunkLarge;  // the documented size limit assumes 16-tile chunks
     a.device_status = device_status;

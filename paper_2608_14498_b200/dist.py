@@ -50,3 +50,39 @@ def job_throughput(local_units: float, local_ms: float, device=None) -> Tuple[fl
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return float(n.item()), float(t.item())
+
+
+def vocab_shard_bounds(vocab: int, world_size: int, rank: int, multiple: int = 256):
+    """[begin, end) of the vocabulary rows rank `rank` holds: equal shares rounded to `multiple`
+    columns (one LM-head tile), the last rank taking the remainder (possibly empty-free: >= 1)."""
+    per = -(-vocab // world_size)
+    per = -(-per // multiple) * multiple
+    begin = min(vocab, rank * per)
+    end = vocab if rank == world_size - 1 else min(vocab, begin + per)
+    return begin, end
+
+
+def gather_shard_stats(stats, group=None):
+    """All ranks' shard records stacked in rank order: [N, 4] per rank -> [world, N, 4].
+
+    This is the one exchange of the vocabulary-parallel LM head (16 bytes per row and rank).
+    Without an initialised process group the result has a single shard."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return stats.unsqueeze(0).contiguous()
+    chunks = [torch.empty_like(stats) for _ in range(dist.get_world_size(group))]
+    dist.all_gather(chunks, stats.contiguous(), group=group)
+    return torch.stack(chunks).contiguous()
+
+
+def vocab_parallel_token_logprobs(hidden, w_shard, target_ids, vocab_begin: int, vocab_total: int, group=None,
+                                  entropy=None, device_status=None):
+    """LM-head log-probs with W_vocab sharded over the ranks of `group` (hidden rows replicated):
+    shard call, one all-gather of the per-row records, merge call."""
+    from . import binding as B
+
+    stats = B.token_logprobs_shard(hidden, w_shard, target_ids, vocab_begin, device_status=device_status)
+    gathered = gather_shard_stats(stats, group)
+    return B.token_logprobs_merge(gathered, target_ids, vocab_total, entropy=entropy, device_status=device_status)

@@ -25,7 +25,14 @@ def _worker(rank: int, world: int, port: int, out):
         cfg = wk.Config("t", "bf16", 4, 4, 2, 64, 64, 128, ("lognormal", 60, 0.5, 8, 200), ("uniform", 1, 30))
         wl = wk.make_workload(cfg, seed=rank, attn=False, lm=False)
         units, ms = rdist.job_throughput(wl.n_tokens, 10.0 * (rank + 1))
-        out.put((rank, wl.n_tokens, units, ms))
+        # the exchange step of the vocabulary-parallel LM head: records stacked in rank order
+        import torch
+        stats = torch.full((5, 4), float(rank + 1)) + torch.arange(5, dtype=torch.float32)[:, None]
+        gathered = rdist.gather_shard_stats(stats)
+        ok = tuple(gathered.shape) == (world, 5, 4) and all(
+            torch.equal(gathered[r], torch.full((5, 4), float(r + 1)) + torch.arange(5, dtype=torch.float32)[:, None])
+            for r in range(world))
+        out.put((rank, wl.n_tokens, units, ms, ok))
         dist.barrier()
     finally:
         dist.destroy_process_group()
@@ -44,12 +51,15 @@ def test_job_throughput_sums_units_and_takes_the_slowest_rank():
         assert p.exitcode == 0
     local = [r[1] for r in res]
     assert local[0] != local[1]  # different seeds, different batches
-    for _, _, units, ms in res:
-        assert units == float(sum(local)) and ms == 20.0
+    for _, _, units, ms, gathered_ok in res:
+        assert units == float(sum(local)) and ms == 20.0 and gathered_ok
 
 
 def test_single_process_job_throughput_is_local():
+    import torch
+
     assert rdist.job_throughput(123, 4.5) == (123.0, 4.5)
+    assert tuple(rdist.gather_shard_stats(torch.zeros(3, 4)).shape) == (1, 3, 4)
 
 
 def test_partition_covers_every_sequence_once_and_balances():
