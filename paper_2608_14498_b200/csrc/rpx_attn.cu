@@ -21,6 +21,8 @@
 // running max grows by more than 2^8).
 #include <math_constants.h>
 
+#include <type_traits>
+
 #include "rpx_internal.h"
 #include "rpx_ptx.cuh"
 
@@ -117,6 +119,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     // load stalls the in-order warp for hundreds of cycles.)
     const int32_t n_tile0 = n_prefix_tiles + 2 * pair + 1;
     const int32_t n_kv = active1 ? n_tile0 + 1 : n_tile0;
+    // Rows that see only a handful of keys (the first rows of a sequence with little or no cached
+    // prefix) get no averaging over keys, so the 2^-9 rounding of each bf16 probability shows up in
+    // O at full size (up to 2^-9 * |v|) and, stacked on the bf16 rounding of O itself, can pass 1e-2.
+    // A query tile that holds such rows has at most two key steps (n_tile0 + t <= 2: the first CTA
+    // of a sequence with at most one tile of cached prefix).  For it the probabilities are kept as
+    // two bf16 terms, P = P_hi + P_lo, with P_lo in the unused upper half of S_t's columns and a
+    // second PV MMA: exact to 2^-17 at the cost of at most four extra MMA groups per sequence and head.
 
     extern __shared__ __align__(1024) uint8_t smem[];
     if ((smem_u32(smem) & 1023u) != 0u) {  // swizzled tiles need 1024-byte alignment; never expected
@@ -309,9 +318,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             };
             auto issue_pv = [&](int t, uint32_t v_slot, bool accumulate) {
                 // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
-                umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128,
-                             v_desc0 + static_cast<uint64_t>(v_slot * (L::kKvBytes >> 4)), idesc_pv,
-                             accumulate ? 1u : 0u);
+                const uint64_t vd = v_desc0 + static_cast<uint64_t>(v_slot * (L::kKvBytes >> 4));
+                umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128, vd, idesc_pv, accumulate ? 1u : 0u);
+                if (n_tile0 + t <= 2)  // + P_lo V, P_lo in columns 64..127 of S_t
+                    umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128 + 64, vd, idesc_pv, 1u);
             };
 
             ok = mbar_wait(&ctl->q_full, 0, abort_flag);
@@ -378,7 +388,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             const uint32_t my_o = tmem_base + 256 + t * 128 + lane_addr;  // and of O_t
             float run_max = -CUDART_INF_F, run_sum = 0.f;
             bool ok = true;
-            for (int32_t j = 0; j < my_tiles; ++j) {
+            // The whole step loop is instantiated twice, so the common (kSplit = false) instance is
+            // scheduled and register-allocated exactly as if the two-term variant did not exist.
+            auto run_steps = [&](auto split_tag) {
+              constexpr bool kSplit = decltype(split_tag)::value;
+              for (int32_t j = 0; j < my_tiles; ++j) {
                 if (!mbar_wait(&ctl->s_full[t], j & 1, abort_flag)) {
                     ok = false;
                     break;
@@ -427,32 +441,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
                 const uint64_t neg_max2 = f2_pack(-run_max, -run_max);
                 uint64_t part2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed accumulators = eight chains
+                // kSplit also writes the second bf16 term of each probability (what the first term's
+                // rounding dropped) to columns 64..127, four words at a time to keep it in registers.
+                {
 #pragma unroll
-                for (int c = 0; c < kChunks; ++c) {
-                    uint32_t packed[16];
+                    for (int c = 0; c < kChunks; ++c) {
+                        uint32_t packed[16];
+                        uint32_t lo[4];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const uint64_t x = f2_fma(f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])),
-                                                  scale2, neg_max2);
-                        float e0, e1;
-                        float x0, x1;
-                        f2_unpack(x, x0, x1);
-                        if (((i / 2) % 4) < kPolyPairsOf4) {  // compile-time per unrolled pair
-                            e0 = poly_exp2(x0);  // scalar form: its constants are immediates, the packed
-                            e1 = poly_exp2(x1);  // form would pin seven register pairs in this loop
-                        } else {
-                            e0 = fast_exp2(x0);
-                            e1 = fast_exp2(x1);
+                        for (int i = 0; i < 32; i += 2) {
+                            const uint64_t x = f2_fma(
+                                f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])), scale2, neg_max2);
+                            float e0, e1;
+                            float x0, x1;
+                            f2_unpack(x, x0, x1);
+                            if (((i / 2) % 4) < kPolyPairsOf4) {  // compile-time per unrolled pair
+                                e0 = poly_exp2(x0);  // scalar form: its constants are immediates, the packed
+                                e1 = poly_exp2(x1);  // form would pin seven register pairs in this loop
+                            } else {
+                                e0 = fast_exp2(x0);
+                                e1 = fast_exp2(x1);
+                            }
+                            part2[(i / 2) % 4] = f2_add(part2[(i / 2) % 4], f2_pack(e0, e1));
+                            const uint32_t hi = pack_bf16x2(e0, e1);
+                            packed[i >> 1] = hi;
+                            if constexpr (kSplit) {
+                                lo[(i >> 1) & 3] = pack_bf16x2(e0 - __uint_as_float(hi << 16),
+                                                               e1 - __uint_as_float(hi & 0xffff0000u));
+                                if (((i >> 1) & 3) == 3) tmem_st4(my_s + 64 + c * 16 + (i >> 1) - 3, lo);
+                            }
                         }
-                        part2[(i / 2) % 4] = f2_add(part2[(i / 2) % 4], f2_pack(e0, e1));
-                        packed[i >> 1] = pack_bf16x2(e0, e1);
+                        tmem_st16(my_s + c * 16, packed);
                     }
-                    tmem_st16(my_s + c * 16, packed);
                 }
                 {
-                    float a0, a1, b0, b1;
+                    float a0, a1;
                     f2_unpack(f2_add(f2_add(part2[0], part2[1]), f2_add(part2[2], part2[3])), a0, a1);
-                    (void)b0; (void)b1;
                     run_sum += a0 + a1;
                 }
                 // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent until this warp's arrival
@@ -474,7 +498,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->p_ready[t]);
-            }
+              }
+            };
+            if (my_tiles <= 2)
+                run_steps(std::true_type{});
+            else
+                run_steps(std::false_type{});
             // ---- epilogue: O / l -> global, LSE
             if (ok) ok = mbar_wait(&ctl->o_done[t], 0, abort_flag);
             if (ok) {

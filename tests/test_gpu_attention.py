@@ -49,16 +49,34 @@ def run_split(wl, dev, table=None, sentinel=SENTINEL):
     return out, lse, bf16_bits(k_cache), bf16_bits(v_cache), (o_pre, o_suf)
 
 
-def check_rows(wl, out, lse, rows, lse_tol=LSE_TOL):
-    ref_o, ref_l = oracle.attn_rows(wl.q, wl.k, wl.v, wl.cu_full, rows)
+def out_tolerance(ref_o):
+    """Element-wise bound on |O_kernel - O_oracle|.
+
+    1e-2 wherever |O| < 4.  The output is stored as bf16, whose half-ulp is 2^-6 = 0.0156 on
+    [4, 8) and doubles per binade, so no bf16 result can promise 1e-2 there: those elements (a
+    handful per million with unit-variance V) get half an ulp plus 2.5e-3 for the kernel's own
+    arithmetic.
+    """
+    a = np.abs(ref_o)
+    half_ulp = np.exp2(np.floor(np.log2(np.maximum(a, 1.0))) - 8.0)
+    return np.where(a < 4.0, TOL, half_ulp + 2.5e-3)
+
+
+def check_rows(wl, out, lse, rows, lse_tol=LSE_TOL, inputs=None):
+    q, k, v = (wl.q, wl.k, wl.v) if inputs is None else inputs
+    ref_o, ref_l = oracle.attn_rows(q, k, v, wl.cu_full, rows)
     tok = wl.cu_full[rows[:, 0]].astype(np.int64) + rows[:, 1]
     got_o, got_l = out[tok, rows[:, 2]], lse[tok, rows[:, 2]]
     assert np.isfinite(got_o).all()
-    err_o = np.abs(got_o - ref_o).max()
-    err_l = np.abs(got_l - ref_l).max()
-    assert err_o <= TOL, f"attention max-abs error {err_o:.3e}"
+    err = np.abs(got_o - ref_o)
+    over = err - out_tolerance(ref_o)
+    err_l = np.abs(got_l - ref_l).max() if rows.shape[0] else 0.0
+    if over.size and over.max() > 0:
+        i, j = np.unravel_index(over.argmax(), over.shape)
+        raise AssertionError(f"attention error {err[i, j]:.3e} at row {rows[i]} col {j}: ref {ref_o[i, j]:.6f} "
+                             f"got {got_o[i, j]:.6f}")
     assert err_l <= lse_tol, f"LSE max-abs error {err_l:.3e}"
-    return err_o, err_l
+    return (err.max() if err.size else 0.0), err_l
 
 
 def check_cache(wl, kc, vc, table=None):
