@@ -6,11 +6,13 @@ or eager fallback: a missing library or a non-sm_100 device is an error.
 """
 from .binding import (  # noqa: F401
     RpxError,
+    get_sm_budget,
     library_path,
     load_library,
     prefix_attn,
     prefix_attn_workspace_bytes,
     selftest_bounded_wait,
+    set_sm_budget,
     status_string,
     suffix_attn,
     suffix_attn_workspace_bytes,

@@ -30,6 +30,8 @@ EXPORTS = (
     "rpx_suffix_attn_workspace_bytes",
     "rpx_token_logprobs_workspace_bytes",
     "rpx_selftest_bounded_wait",
+    "rpx_set_sm_budget",
+    "rpx_get_sm_budget",
     "rpx_status_string",
     "rpx_version",
 )
@@ -102,6 +104,10 @@ def load_library():
     lib.rpx_token_logprobs_workspace_bytes.argtypes = [i64, i32, i32, i32]
     lib.rpx_selftest_bounded_wait.restype = i32
     lib.rpx_selftest_bounded_wait.argtypes = [i64, vp, vp]
+    lib.rpx_set_sm_budget.restype = i32
+    lib.rpx_set_sm_budget.argtypes = [i32]
+    lib.rpx_get_sm_budget.restype = i32
+    lib.rpx_get_sm_budget.argtypes = []
     lib.rpx_status_string.restype = ctypes.c_char_p
     lib.rpx_status_string.argtypes = [i32]
     lib.rpx_version.restype = i32
@@ -198,6 +204,17 @@ def selftest_bounded_wait(limit_cycles: int, device_status, stream=None) -> None
     rc = load_library().rpx_selftest_bounded_wait(int(limit_cycles), _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
         raise RpxError(rc, "rpx_selftest_bounded_wait")
+
+
+def set_sm_budget(sms: int) -> None:
+    """rpx_set_sm_budget: cap the persistent LM-head grid at ``sms`` CTAs (0 = no cap), process-wide."""
+    rc = load_library().rpx_set_sm_budget(int(sms))
+    if rc != 0:
+        raise RpxError(rc, "rpx_set_sm_budget")
+
+
+def get_sm_budget() -> int:
+    return int(load_library().rpx_get_sm_budget())
 
 
 # ------------------------------------------------------------------ the three calls

@@ -16,6 +16,10 @@ under 19 % active SMs for it).  The stand-in is torch.mv — it is the interferi
 part of the scoring path.  Reported per decode length: T_D, T_P alone, both under co-run, Delta_D,
 the measured saving S = T_D + T_P - makespan and Eq. 1's S from the measured Delta_D and the
 standalone T_P (the model has no term for the prefix work's own slowdown; the difference shows it).
+
+``--sm-budgets`` repeats the measurement with the persistent LM-head grid capped at that many CTAs
+(``rpx_set_sm_budget``; 0 = all SMs), which is how a caller leaves the decode side room: T_P grows
+by about SMs/budget, Delta_D shrinks.
 """
 from __future__ import annotations
 
@@ -38,6 +42,7 @@ def main() -> None:
     ap.add_argument("--ratios", type=float, nargs="+", default=[0.5, 1.0, 2.0], help="target T_D / T_P")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--decode-gb", type=float, default=4.0, help="weight bytes one decode step streams")
+    ap.add_argument("--sm-budgets", type=int, nargs="+", default=[0], help="LM-head CTA caps to sweep (0 = none)")
     args = ap.parse_args()
     dev = torch.device("cuda", 0)
     B.load_library()
@@ -100,28 +105,31 @@ def main() -> None:
 
     for _ in range(3):
         timed(True, 4)
-    t_p, _ = median(True, 0)
     _, t_step = median(False, 16)
     t_step /= 16
-    sess.check_status()
-    for ratio in args.ratios:
-        steps = max(1, round(ratio * t_p / t_step))
-        _, t_d = median(False, steps)
-        t_p_co, t_d_co = median(True, steps)
-        delta_d = t_d_co - t_d
-        makespan = max(t_d_co, t_p_co)
-        line = {
-            "experiment": "corun_eq1", "workload": cfg.name, "decode_steps": steps,
-            "decode_step_bytes": rows * cols * 2, "T_D_ms": t_d, "T_P_ms": t_p, "T_D_corun_ms": t_d_co,
-            "T_P_corun_ms": t_p_co, "Delta_D_ms": delta_d, "Delta_D_pct": 100.0 * delta_d / t_d,
-            "prefix_slowdown_pct": 100.0 * (t_p_co - t_p) / t_p,
-            "S_measured_ms": t_d + t_p - makespan,
-            # Eq. 1 with the measured Delta_D; it charges interference to decode only, so the gap to
-            # S_measured is the prefix work's own slowdown under co-run
-            "S_eq1_ms": t_d + t_p - max(t_d + delta_d, t_p),
-            "serial_ms": t_d + t_p, "overlapped_ms": makespan, "speedup": (t_d + t_p) / makespan,
-        }
-        print(json.dumps(line), flush=True)
+    for budget in args.sm_budgets:
+        B.set_sm_budget(budget)
+        t_p, _ = median(True, 0)
+        sess.check_status()
+        for ratio in args.ratios:
+            steps = max(1, round(ratio * t_p / t_step))
+            _, t_d = median(False, steps)
+            t_p_co, t_d_co = median(True, steps)
+            delta_d = t_d_co - t_d
+            makespan = max(t_d_co, t_p_co)
+            line = {
+                "experiment": "corun_eq1", "workload": cfg.name, "sm_budget": budget, "decode_steps": steps,
+                "decode_step_bytes": rows * cols * 2, "T_D_ms": t_d, "T_P_ms": t_p, "T_D_corun_ms": t_d_co,
+                "T_P_corun_ms": t_p_co, "Delta_D_ms": delta_d, "Delta_D_pct": 100.0 * delta_d / t_d,
+                "prefix_slowdown_pct": 100.0 * (t_p_co - t_p) / t_p,
+                "S_measured_ms": t_d + t_p - makespan,
+                # Eq. 1 with the measured Delta_D; it charges interference to decode only, so the gap to
+                # S_measured is the prefix work's own slowdown under co-run
+                "S_eq1_ms": t_d + t_p - max(t_d + delta_d, t_p),
+                "serial_ms": t_d + t_p, "overlapped_ms": makespan, "speedup": (t_d + t_p) / makespan,
+            }
+            print(json.dumps(line), flush=True)
+    B.set_sm_budget(0)
     sess.check_status()
 
 

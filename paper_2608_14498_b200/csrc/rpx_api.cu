@@ -274,6 +274,14 @@ const char* rpx_status_string(rpx_status_t status) {
     }
 }
 
+rpx_status_t rpx_set_sm_budget(int32_t sms) {
+    if (sms < 0) return RPX_ERR_SHAPE;
+    rpx::set_sm_budget(sms);
+    return RPX_OK;
+}
+
+int32_t rpx_get_sm_budget(void) { return rpx::sm_budget(); }
+
 int32_t rpx_version(void) { return 100; }
 
 }  // extern "C"

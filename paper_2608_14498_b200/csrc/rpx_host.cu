@@ -2,6 +2,7 @@
 // queries, and the fp32 -> bf16 pre-pass used for RPX_F32 inputs.
 #include <cuda_bf16.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "rpx_internal.h"
@@ -85,6 +86,12 @@ int sm_count() {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
     return n;
 }
+
+namespace {
+std::atomic<int> g_sm_budget{0};
+}
+int sm_budget() { return g_sm_budget.load(std::memory_order_relaxed); }
+void set_sm_budget(int sms) { g_sm_budget.store(sms, std::memory_order_relaxed); }
 
 rpx_status_t check_arch() {
     int dev = 0, major = 0;

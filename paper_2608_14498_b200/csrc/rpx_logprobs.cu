@@ -340,8 +340,9 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     const int64_t total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
     if (total > INT32_MAX) return RPX_ERR_SHAPE;
     p.total_items = static_cast<int32_t>(total);
-    const int sms = sm_count();
+    int sms = sm_count();
     if (sms <= 0) return RPX_ERR_CUDA;
+    if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;  // leave the rest to a co-runner
     const int grid = static_cast<int>(total < sms ? total : sms);
     p.group_width = (grid % 4 == 0) ? 4 : (grid % 2 == 0 ? 2 : 1);
     p.target_ids = a.target_ids;

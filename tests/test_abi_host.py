@@ -39,6 +39,17 @@ def test_version_and_status_strings(lib):
     assert B.status_string(-99) == "unknown status"
 
 
+def test_sm_budget_is_host_state_with_validation(lib):
+    assert B.get_sm_budget() == 0
+    B.set_sm_budget(96)
+    assert B.get_sm_budget() == 96
+    with pytest.raises(B.RpxError) as e:
+        B.set_sm_budget(-1)
+    assert e.value.status == -2 and B.get_sm_budget() == 96  # rejected, unchanged
+    B.set_sm_budget(0)
+    assert B.get_sm_budget() == 0
+
+
 def test_workspace_arithmetic(lib):
     assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 32768) == 0
     need = B.prefix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 256)

@@ -101,6 +101,22 @@ def test_two_calls_give_identical_bits(cuda_device):
     assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("budget", [1, 37, 100, 1000])
+def test_sm_budget_changes_no_bit(cuda_device, budget):
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, 256, 70000, ("fixed", 3000), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=8, attn=False)
+    h, w, ids = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    a = rpx.token_logprobs(h, w, ids).clone()
+    try:
+        rpx.set_sm_budget(budget)
+        b = rpx.token_logprobs(h, w, ids)
+        torch.cuda.synchronize()
+    finally:
+        rpx.set_sm_budget(0)
+    assert torch.equal(a, b)
+
+
 def test_c2_full_size_sampled_rows(cuda_device):
     """BASELINE configs[1] at full size (34 816 rows x 152 064 columns, hidden 3584), in the launch
     configuration the benchmark times; the oracle scores 48 sampled rows one by one."""
