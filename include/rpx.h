@@ -127,6 +127,28 @@ RPX_API rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q,
                              size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
 /*
+ * Chunked prefill of the prefix (an extension: the paper prefills each prompt in one pass and only
+ * fixes a per-prompt token budget, Section 4.1).  One call handles the next chunk of every prompt:
+ * chunk position i of sequence s (global position cached_lens[s] + i) attends to the cached_lens[s]
+ * keys already in the cache and to chunk keys 0..i, exactly as rpx_suffix_attn does, AND the
+ * chunk's K and V are appended to the cache at global positions cached_lens[s] + i, exactly as
+ * rpx_prefix_attn stores them.  After the last chunk the cache and the concatenated outputs equal
+ * those of one rpx_prefix_attn call over the whole prompts.
+ *   cached_lens device int32 [batch]: tokens already cached; each must be a multiple of the
+ *   block size (chunks start on a page edge) — otherwise nothing is stored for that sequence and
+ *   RPX_ERR_DEVICE_DATA appears in *device_status (its attention rows are still computed).
+ *   The block table must cover cached_lens[s] + chunk length.  A sequence whose chunk is empty
+ *   (cu_seqlens_chunk[s] == cu_seqlens_chunk[s+1]) is skipped whatever its cached_lens.
+ *   Other arguments as rpx_suffix_attn; workspace as rpx_suffix_attn_workspace_bytes.
+ */
+RPX_API rpx_status_t rpx_chunk_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                            int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,
+                            const int32_t* cu_seqlens_chunk, const int32_t* cached_lens, int32_t batch,
+                            int64_t total_chunk_tokens, int32_t max_chunk_len, int32_t max_cached_len,
+                            const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
+/*
  * Fused LM-head log-probabilities (Section 3.1: Phase 1 yields "prefix log-probabilities",
  * Phase 2 the suffix ones; Table 4 "Prefix logprobs").  For every row n:
  *     z_v = hidden[n,:] . w_vocab[v,:]          (never stored)

@@ -6,6 +6,7 @@ or eager fallback: a missing library or a non-sm_100 device is an error.
 """
 from .binding import (  # noqa: F401
     RpxError,
+    chunk_attn,
     get_sm_budget,
     library_path,
     load_library,

@@ -21,6 +21,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "rpx_prefix_attn",
     "rpx_suffix_attn",
+    "rpx_chunk_attn",
     "rpx_token_logprobs",
     "rpx_token_logprobs_entropy",
     "rpx_token_logprobs_shard",
@@ -85,6 +86,9 @@ def load_library():
                                     ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
     lib.rpx_suffix_attn.restype = i32
     lib.rpx_suffix_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, i64, i64, i64, vp, vp, i32, i64, i32,
+                                    i32, ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
+    lib.rpx_chunk_attn.restype = i32
+    lib.rpx_chunk_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, i64, i64, i64, vp, vp, i32, i64, i32,
                                     i32, ctypes.POINTER(KvCache), vp, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs.restype = i32
     lib.rpx_token_logprobs.argtypes = [vp, i64, vp, vp, i64, i32, i32, i32, vp, vp, vp, sz, vp, vp]
@@ -265,6 +269,31 @@ def suffix_attn(q, k, v, cu_seqlens_suffix, prefix_lens, max_suffix_len: int, ma
                              _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
         raise RpxError(rc, "rpx_suffix_attn")
+    return (out, lse) if return_lse else out
+
+
+def chunk_attn(q, k, v, cu_seqlens_chunk, cached_lens, max_chunk_len: int, max_cached_len: int, cache: Tuple,
+                softmax_scale: float = 0.0, out=None, lse=None, return_lse: bool = False, workspace=None,
+                device_status=None, stream=None):
+    """rpx_chunk_attn: the next chunk of every prompt over [cached earlier chunks ; causal self], appending
+    the chunk's K/V to the cache (cached_lens must be multiples of the 16-token block)."""
+    torch = _torch()
+    lib = load_library()
+    desc = _desc(q, k, softmax_scale)
+    total = q.shape[0]
+    if out is None:
+        out = torch.empty((total, q.shape[1], q.shape[2]), dtype=q.dtype, device=q.device)
+    if lse is None and return_lse:
+        lse = torch.empty((total, q.shape[1]), dtype=torch.float32, device=q.device)
+    ws = _workspace(int(lib.rpx_suffix_attn_workspace_bytes(ctypes.byref(desc), total)), q.device, workspace)
+    cs = _cache_struct(cache)
+    rc = lib.rpx_chunk_attn(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _tok_stride(q), _tok_stride(k),
+                             _tok_stride(v), _ptr(cu_seqlens_chunk), _ptr(cached_lens),
+                             cu_seqlens_chunk.shape[0] - 1, total, int(max_chunk_len), int(max_cached_len),
+                             ctypes.byref(cs), _ptr(out), _ptr(lse), _ptr(ws), ws.numel() * ws.element_size(),
+                             _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_chunk_attn")
     return (out, lse) if return_lse else out
 
 

@@ -38,7 +38,7 @@ rpx_status_t check_cache(const rpx_kv_cache_t* c, int32_t batch) {
 // Shared body of the two attention entry points.  prefix_lens == NULL selects the prefix pass.
 rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
                            int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const int32_t* cu_seqlens,
-                           const int32_t* prefix_lens, bool is_suffix, int32_t batch, int64_t total_tokens,
+                           const int32_t* prefix_lens, bool is_suffix, bool append_cache, int32_t batch, int64_t total_tokens,
                            int32_t max_q_len, int32_t max_prefix_len, const rpx_kv_cache_t* cache, void* out, float* lse,
                            void* workspace, size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
     if (rpx_status_t rc = check_attn_desc(desc)) return rc;
@@ -98,6 +98,7 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.max_q_len = max_q_len;
     a.max_prefix_len = max_prefix_len;
     a.cache = cache;
+    a.append_cache = is_suffix && append_cache;
     a.out = out;
     a.out_f32 = desc->dtype == RPX_F32;
     a.lse = lse;
@@ -115,7 +116,7 @@ rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const v
                              const int32_t* cu_seqlens, int32_t batch, int64_t total_tokens, int32_t max_seqlen,
                              const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
-    return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens, nullptr, false, batch,
+    return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens, nullptr, false, false, batch,
                          total_tokens, max_seqlen, 0, cache, out, lse, workspace, workspace_bytes, device_status,
                          cuda_stream);
 }
@@ -127,12 +128,22 @@ rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const v
                              const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
     return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens_suffix, prefix_lens, true,
-                         batch, total_suffix_tokens, max_suffix_len, max_prefix_len, cache, out, lse, workspace,
+                         false, batch, total_suffix_tokens, max_suffix_len, max_prefix_len, cache, out, lse, workspace,
                          workspace_bytes, device_status, cuda_stream);
 }
 
 size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens) {
     return attn_workspace(desc, total_tokens);
+}
+
+rpx_status_t rpx_chunk_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                            int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const int32_t* cu_seqlens_chunk,
+                            const int32_t* cached_lens, int32_t batch, int64_t total_chunk_tokens, int32_t max_chunk_len,
+                            int32_t max_cached_len, const rpx_kv_cache_t* cache, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+    return run_attention(desc, q, k, v, q_tok_stride, k_tok_stride, v_tok_stride, cu_seqlens_chunk, cached_lens, true,
+                         true, batch, total_chunk_tokens, max_chunk_len, max_cached_len, cache, out, lse, workspace,
+                         workspace_bytes, device_status, cuda_stream);
 }
 
 size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens) {

@@ -79,7 +79,7 @@ struct Params {
     int64_t num_blocks;
     __nv_bfloat16* k_cache;       // used by the ragged-page paths
     __nv_bfloat16* v_cache;
-    int32_t write_cache;          // prefix pass with a cache
+    int32_t write_cache;          // store this call's K/V into the cache (prefix pass, chunked prefill)
     int32_t batch, num_q_heads, num_kv_heads, group;
     int32_t n_pairs;              // query tile pairs per sequence the grid covers
     float scale_log2;
@@ -177,7 +177,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     tma_load_3d(smem + L::kQOff + t * L::kQBytes + hf * L::kHalfBytes, &tmap_q, &ctl->q_full,
                                 hf * 64, head, tok0 + q0 + t * kTileQ);
         }
-        const bool owns_cache_write = p.write_cache != 0 && (head % p.group) == 0;
+        // Appending behind a cached prefix (chunked prefill) needs the chunk to start on a page edge:
+        // pages are written whole or from their first row.  Anything else is reported, not written.
+        const bool page_aligned = (len_p % kPage) == 0;
+        if (p.write_cache != 0 && !page_aligned && lane == 0) ctl->data_error = 1;
+        const bool owns_cache_write = p.write_cache != 0 && page_aligned && (head % p.group) == 0;
+        const int32_t write_page0 = len_p / kPage;  // first page of this call's own tokens
         uint32_t n_loaded = 0;
         for (int32_t j = 0; ok && j < n_kv; ++j) {
             const bool from_cache = j < n_prefix_tiles;
@@ -256,7 +261,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     const int32_t n_pages = (rows_valid + kPage - 1) / kPage;
                     int32_t blk = 0;
                     if (lane < n_pages) {
-                        blk = p.block_table[static_cast<int64_t>(seq) * p.block_table_stride + jt * (kTileK / kPage) + lane];
+                        blk = p.block_table[static_cast<int64_t>(seq) * p.block_table_stride + write_page0 +
+                                            jt * (kTileK / kPage) + lane];
                         if (blk < 0 || blk >= p.num_blocks) {
                             ctl->data_error = 1;
                             blk = -1;
@@ -592,7 +598,7 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.num_blocks = a.cache ? a.cache->num_blocks : 0;
     p.k_cache = a.cache ? static_cast<__nv_bfloat16*>(a.cache->k_cache) : nullptr;
     p.v_cache = a.cache ? static_cast<__nv_bfloat16*>(a.cache->v_cache) : nullptr;
-    p.write_cache = (a.cache != nullptr && a.prefix_lens == nullptr) ? 1 : 0;
+    p.write_cache = (a.cache != nullptr && (a.prefix_lens == nullptr || a.append_cache)) ? 1 : 0;
     p.batch = a.batch;
     p.num_q_heads = a.num_q_heads;
     p.num_kv_heads = a.num_kv_heads;

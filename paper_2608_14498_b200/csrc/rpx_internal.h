@@ -37,6 +37,7 @@ struct AttnArgs {
     int64_t total_tokens;
     int32_t max_q_len, max_prefix_len;
     const rpx_kv_cache_t* cache;       // prefix pass: written (nullable); suffix pass: read
+    bool append_cache = false;         // chunked prefill: read the earlier chunks AND append this one
     void* out;
     bool out_f32;
     float* lse;

@@ -93,6 +93,14 @@ def test_attention_rejects_bad_arguments_before_any_launch(lib):
     rc = lib.rpx_suffix_attn(ctypes.byref(good), 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, 0x1000, 1, 16, 16, 64,
                              None, 0x1000, None, None, 0, None, None)
     assert rc == -1
+    # and so does chunked prefill
+    rc = lib.rpx_chunk_attn(ctypes.byref(good), 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, 0x1000, 1, 16, 16, 64,
+                            None, 0x1000, None, None, 0, None, None)
+    assert rc == -1
+    ok_cache = B.KvCache(0x1000, 0x1000, 8, 16, 0x1000, 4)
+    rc = lib.rpx_chunk_attn(ctypes.byref(good), 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, None, 1, 16, 16, 64,
+                            ctypes.byref(ok_cache), 0x1000, None, None, 0, None, None)
+    assert rc == -1  # cached_lens missing
 
 
 def test_logprobs_rejects_bad_arguments_before_any_launch(lib):
