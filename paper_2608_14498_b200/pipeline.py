@@ -67,9 +67,10 @@ class ScoringSession:
         self.v_cache = torch.zeros_like(self.k_cache)
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self._ws = {}
-        self._staging: Optional[Batch] = None
+        self._staging = [None, None]       # two device staging sets: the next pass uploads while this one computes
+        self._staging_free = [None, None]  # event: the pass that used the set has finished reading it
+        self._staging_turn = 0
         self._copy_stream = None
-        self._staging_free = None
         self.kernels_last_host_pass = 0
         self._out = {}
 
@@ -133,19 +134,25 @@ class ScoringSession:
         kernel waits only for its own inputs: the prompt rows of the LM head (the longest kernel)
         are cut into ``lm_slices`` row slices so that scoring starts after the first slice has
         landed and the remaining copies hide behind it.  Kernels and the device->host copy of the
-        results are enqueued on the current stream; the caller synchronises."""
+        results are enqueued on the current stream; the caller synchronises.  Two staging sets
+        alternate, so back-to-back calls overlap one pass's uploads with the previous pass's kernels."""
         t = self.torch
-        if self._staging is None or any(tuple(a.shape) != tuple(c.shape) or a.dtype != c.dtype
-                                        for a, c in zip(self._staging.tensors(), hb.tensors())):
-            dev = [t.empty(x.shape, dtype=x.dtype, device=self.device) for x in hb.tensors()]
-            self._staging = Batch(*dev, hb.max_prefix_len, hb.max_suffix_len)
+        turn = self._staging_turn
+        self._staging_turn ^= 1
+        if self._copy_stream is None:
             self._copy_stream = t.cuda.Stream(device=self.device)
-            self._staging_free = None
-        d = self._staging
         main = t.cuda.current_stream()
         copy = self._copy_stream
-        if self._staging_free is not None:
-            copy.wait_event(self._staging_free)  # last pass has finished reading the staging buffers
+        cur = self._staging[turn]
+        if cur is None or any(tuple(a.shape) != tuple(c.shape) or a.dtype != c.dtype
+                              for a, c in zip(cur.tensors(), hb.tensors())):
+            dev = [t.empty(x.shape, dtype=x.dtype, device=self.device) for x in hb.tensors()]
+            self._staging[turn] = Batch(*dev, hb.max_prefix_len, hb.max_suffix_len)
+            self._staging_free[turn] = None
+        d = self._staging[turn]
+        d.max_prefix_len, d.max_suffix_len = hb.max_prefix_len, hb.max_suffix_len
+        if self._staging_free[turn] is not None:
+            copy.wait_event(self._staging_free[turn])  # the pass before last has finished reading this set
         else:
             copy.wait_stream(main)
 
@@ -158,7 +165,11 @@ class ScoringSession:
             return ev
 
         n_p = hb.hidden_p.shape[0]
-        bounds = [n_p * i // lm_slices for i in range(lm_slices + 1)] if n_p > 0 else [0, 0]
+        # a short first slice (1/16 of the rows) gets the first kernel going early; the rest is cut evenly
+        first = min(n_p, -(-(n_p // 16) // 128) * 128) if lm_slices > 1 else n_p
+        rest = max(lm_slices - 1, 1)
+        bounds = [0] + [first + (n_p - first) * i // rest for i in range(rest + 1)] if n_p > 0 else [0, 0]
+        bounds = sorted(set(bounds)) if n_p > 0 else bounds
         ev_ids = upload([(d.ids_p, hb.ids_p)])
         ev_slices = [upload([(d.hidden_p[a:b], hb.hidden_p[a:b])]) for a, b in zip(bounds[:-1], bounds[1:])]
         ev_prefix = upload([(d.q_p, hb.q_p), (d.k_p, hb.k_p), (d.v_p, hb.v_p), (d.cu_prefix, hb.cu_prefix),
@@ -191,8 +202,8 @@ class ScoringSession:
         B.suffix_attn(d.q_s, d.k_s, d.v_s, d.cu_suffix, d.prefix_lens, d.max_suffix_len, d.max_prefix_len, cache=cache,
                       out=o_s, workspace=attn_ws, device_status=self.status)
         B.token_logprobs(d.hidden_s, self.w_vocab, d.ids_s, logprobs=lp_s, workspace=lm_ws, device_status=self.status)
-        self._staging_free = t.cuda.Event()
-        self._staging_free.record(main)
+        self._staging_free[turn] = t.cuda.Event()
+        self._staging_free[turn].record(main)
         lp_p_host.copy_(lp_p, non_blocking=True)
         lp_s_host.copy_(lp_s, non_blocking=True)
         self.kernels_last_host_pass = 2 + 2 * (sum(1 for a, b in zip(bounds[:-1], bounds[1:]) if b > a) + 1)
