@@ -184,10 +184,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         const bool owns_cache_write = p.write_cache != 0 && page_aligned && (head % p.group) == 0;
         const int32_t write_page0 = len_p / kPage;  // first page of this call's own tokens
         uint32_t n_loaded = 0;
+        // Block id of page `lane` of cached tile jt (lanes 0..7; 0 where the prefix has no such page).
+        // Read one tile ahead, so the table's global-memory latency is off the ring's critical path.
+        auto read_block_ids = [&](int32_t jt) -> int32_t {
+            int32_t b = 0;
+            const int32_t page = jt * (kTileK / kPage) + lane;
+            if (lane < kTileK / kPage && page < (len_p + kPage - 1) / kPage)
+                b = __ldg(p.block_table + static_cast<int64_t>(seq) * p.block_table_stride + page);
+            return b;
+        };
+        int32_t blk_next = n_prefix_tiles > 0 ? read_block_ids(0) : 0;
         for (int32_t j = 0; ok && j < n_kv; ++j) {
             const bool from_cache = j < n_prefix_tiles;
             const int32_t jt = from_cache ? j : j - n_prefix_tiles;  // tile index inside its key source
             uint32_t slot_k = 0, slot_v = 0;
+            int32_t blk = blk_next;  // this tile's pages (cached tiles only)
+            if (from_cache) {
+                if (blk < 0 || blk >= p.num_blocks) {
+                    ctl->data_error = 1;
+                    blk = 0;
+                }
+                if (j + 1 < n_prefix_tiles) blk_next = read_block_ids(j + 1);
+            }
             for (int which = 0; which < 2; ++which, ++n_loaded) {  // 0 = K, 1 = V
                 const uint32_t slot = n_loaded % kSlots, phase = (n_loaded / kSlots) & 1u;
                 if (which == 0) slot_k = slot; else slot_v = slot;
@@ -209,14 +227,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     // meet a non-finite stale V row)
                     const int32_t rows_valid = min(kTileK, len_p - jt * kTileK);
                     const int32_t full_pages = rows_valid / kPage;
-                    int32_t blk = 0;
-                    if (lane <= full_pages && lane < kTileK / kPage && jt * (kTileK / kPage) + lane < (len_p + kPage - 1) / kPage) {
-                        blk = p.block_table[static_cast<int64_t>(seq) * p.block_table_stride + jt * (kTileK / kPage) + lane];
-                        if (blk < 0 || blk >= p.num_blocks) {
-                            ctl->data_error = 1;
-                            blk = 0;
-                        }
-                    }
                     if (full_pages < kTileK / kPage) {
                         const int32_t blk_r = __shfl_sync(0xffffffffu, blk, full_pages);
                         const __nv_bfloat16* src_pool = which == 0 ? p.k_cache : p.v_cache;
@@ -232,17 +242,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         }
                         fence_proxy_async_smem();
                     }
-                    __syncwarp();
-                    for (int32_t pg = 0; pg < full_pages; ++pg) {
-                        const int32_t b = __shfl_sync(0xffffffffu, blk, pg);
-                        if (lane == 0) {
-                            if (pg == 0) mbar_arrive_expect_tx(&ctl->kv_full[slot], full_pages * kPage * D * 2);
-                            for (int hf = 0; hf < L::kHalves; ++hf)
-                                tma_load_4d(dst + hf * L::kHalfBytes + pg * (kPage * 128), which == 0 ? &tmap_kc : &tmap_vc,
-                                            &ctl->kv_full[slot], hf * 64, 0, kv_head, b);
-                        }
+                    if (lane == 0) {
+                        if (full_pages > 0) mbar_arrive_expect_tx(&ctl->kv_full[slot], full_pages * kPage * D * 2);
+                        else mbar_arrive(&ctl->kv_full[slot]);
                     }
-                    if (full_pages == 0 && lane == 0) mbar_arrive(&ctl->kv_full[slot]);
+                    __syncwarp();  // the byte count is armed before any copy can complete
+                    if (lane < full_pages) {  // lane pg fetches page pg (it holds that page's block id)
+                        for (int hf = 0; hf < L::kHalves; ++hf)
+                            tma_load_4d(dst + hf * L::kHalfBytes + lane * (kPage * 128), which == 0 ? &tmap_kc : &tmap_vc,
+                                        &ctl->kv_full[slot], hf * 64, 0, kv_head, blk);
+                    }
                 }
                 __syncwarp();
             }
