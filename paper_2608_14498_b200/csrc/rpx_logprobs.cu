@@ -2,8 +2,8 @@
 //
 //   logprob[n] = z[n, target[n]] - ln sum_v exp(z[n, v]),   z = hidden . W_vocab^T  (never stored)
 //
-// One persistent CTA per SM.  A work item is (row tile of 128 rows, chunk of 16 (4 for small row
-// counts) vocab tiles of 256 columns): the CTA sweeps the chunk tile by tile; each tile is a TMA-fed tcgen05
+// One persistent CTA per SM.  A work item is (row tile of 128 rows, chunk of 16 (4 for small, 8 for very
+// large row counts) vocab tiles of 256 columns): the CTA sweeps the chunk tile by tile; each tile is a TMA-fed tcgen05
 // GEMM over the hidden dimension into one of two 128x256 fp32 TMEM accumulators, and while the
 // tensor core fills one accumulator the four epilogue warps fold the other into a running
 // (max, sum-exp, target-logit) per row.  One partial per (chunk, row) goes to the workspace; a
@@ -27,7 +27,10 @@ namespace {
 constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
 constexpr int kTilesPerChunkLarge = 16;  // many row tiles: long items, few partial records
 constexpr int kTilesPerChunkSmall = 4;   // few row tiles: short items, so the last wave is short too
+constexpr int kTilesPerChunkHuge = 8;    // very many row tiles: there are enough items per CTA that halving
+                                         // them costs nothing and evens out the last wave (measured +1 %)
 constexpr int kSmallRowTiles = 64;
+constexpr int kHugeRowTiles = 192;
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
@@ -306,7 +309,9 @@ __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int3
 }  // namespace
 
 int32_t logprob_tiles_per_chunk(int64_t n_tokens) {
-    return (n_tokens + kBM - 1) / kBM <= kSmallRowTiles ? kTilesPerChunkSmall : kTilesPerChunkLarge;
+    const int64_t row_tiles = (n_tokens + kBM - 1) / kBM;
+    if (row_tiles <= kSmallRowTiles) return kTilesPerChunkSmall;
+    return row_tiles >= kHugeRowTiles ? kTilesPerChunkHuge : kTilesPerChunkLarge;
 }
 
 int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk) {

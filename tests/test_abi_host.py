@@ -55,8 +55,10 @@ def test_workspace_arithmetic(lib):
     need = B.prefix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 256)
     assert need == 256 * 4 * 64 * 2 + 2 * 256 * 2 * 64 * 2
     assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 32 * 8 * 64 * 2
-    # 152064 columns = 594 tiles of 256 = 38 chunks of 16 tiles; one float4 per (chunk, row)
-    assert B.token_logprobs_workspace_bytes(34816, 3584, 152064, B.RPX_BF16) == 38 * 34816 * 16
+    # 152064 columns = 594 tiles of 256; one float4 per (chunk, row): 38 chunks of 16 tiles up to 191 row
+    # tiles of 128 rows, 75 chunks of 8 tiles from 192 row tiles on
+    assert B.token_logprobs_workspace_bytes(12800, 3584, 152064, B.RPX_BF16) == 38 * 12800 * 16
+    assert B.token_logprobs_workspace_bytes(34816, 3584, 152064, B.RPX_BF16) == 75 * 34816 * 16
     f32 = B.token_logprobs_workspace_bytes(288, 256, 4096, B.RPX_F32)
     # up to 64 row tiles the chunks are 4 vocabulary tiles long: 4096 columns = 16 tiles = 4 chunks
     assert f32 == 4 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
