@@ -349,7 +349,10 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     if (sms <= 0) return RPX_ERR_CUDA;
     if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;  // leave the rest to a co-runner
     const int grid = static_cast<int>(total < sms ? total : sms);
-    p.group_width = (grid % 4 == 0) ? 4 : (grid % 2 == 0 ? 2 : 1);
+    // vocab chunks swept side by side by the resident CTAs: 4 keeps (grid / 4) row tiles of hidden states
+    // L2-resident while each W tile is shared by that many CTAs (2 and 8 measured 3 % slower at 256 row
+    // tiles); with few row tiles 2 is 3 % faster
+    p.group_width = (grid % 4 == 0 && p.n_row_tiles > kSmallRowTiles) ? 4 : (grid % 2 == 0 ? 2 : 1);
     p.target_ids = a.target_ids;
     p.target_offset = a.target_offset;
     p.partials = static_cast<float4*>(a.partials);
