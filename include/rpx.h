@@ -100,7 +100,9 @@ typedef struct {
  *   q [total_tokens][num_q_heads][head_dim], k, v [total_tokens][num_kv_heads][head_dim]
  *   out [total_tokens][num_q_heads][head_dim] contiguous, element type desc->dtype
  *   lse (nullable) float32 [total_tokens][num_q_heads]: ln sum_j exp(scale * q.k_j)
- *   max_seqlen: an upper bound on the longest sequence (sizes the grid).
+ *   max_seqlen: an upper bound on the longest sequence (sizes the grid).  A sequence longer than
+ *   the bound rounded up to 256 gets RPX_ERR_DEVICE_DATA in *device_status (its rows beyond the
+ *   bound are not computed); the same holds for max_suffix_len / max_chunk_len below.
  */
 RPX_API rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
                              int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride,

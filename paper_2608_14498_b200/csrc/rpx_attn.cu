@@ -110,6 +110,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     const int32_t tok0 = p.cu_seqlens[seq];
     const int32_t len_q = p.cu_seqlens[seq + 1] - tok0;
     const int32_t q0 = pair * 2 * kTileQ;
+    // A sequence longer than the caller's bound would leave rows the grid never reaches: report it.
+    if (pair == 0 && threadIdx.x == 0 && head == 0 && len_q > p.n_pairs * 2 * kTileQ && p.status != nullptr)
+        atomicCAS(p.status, 0, RPX_ERR_DEVICE_DATA);
     if (q0 >= len_q) return;  // uniform for the whole CTA, before any barrier or allocation
     const int32_t len_p = p.prefix_lens != nullptr ? p.prefix_lens[seq] : 0;
     const bool active1 = q0 + kTileQ < len_q;

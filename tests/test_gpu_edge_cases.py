@@ -115,3 +115,22 @@ def test_strided_fp32_inputs(cuda_device):
     print("fp32-input attention error vs unrounded oracle:", np.abs(got - ref).max())
     assert np.abs(got - ref).max() <= 2.6e-2
     assert np.abs(got_l - ref_l).max() <= 2.6e-2
+
+
+def test_a_sequence_longer_than_the_callers_bound_is_reported(cuda_device):
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 2, 2, 1, 64, 64, 64, ("list", [100, 600]), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=41, lm=False)
+    q, k, v = (to_device(t, dev) for t in (wl.q, wl.k, wl.v))
+    cu = to_device(wl.cu_full, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rpx.prefix_attn(q, k, v, cu, 600, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rpx.prefix_attn(q, k, v, cu, 500, device_status=status)  # rounds up to 512 < 600
+    torch.cuda.synchronize()
+    assert int(status.item()) == -8
+    status.zero_()
+    rpx.prefix_attn(q, k, v, cu, 513, device_status=status)  # rounds up to 768: fine
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
