@@ -20,11 +20,13 @@ rpx_status_t check_attn_desc(const rpx_attn_desc_t* d) {
     return RPX_OK;
 }
 
+// Layout: [work-item counter, kWsAlign bytes][RPX_F32 only: bf16 copies of q, k, v]
 size_t attn_workspace(const rpx_attn_desc_t* d, int64_t tokens) {
-    if (d == nullptr || d->dtype != RPX_F32 || tokens <= 0) return 0;
+    if (d == nullptr || tokens <= 0) return 0;
+    if (d->dtype != RPX_F32) return kWsAlign;
     const size_t qb = align_up(static_cast<size_t>(tokens) * d->num_q_heads * d->head_dim * 2, kWsAlign);
     const size_t kb = align_up(static_cast<size_t>(tokens) * d->num_kv_heads * d->head_dim * 2, kWsAlign);
-    return qb + 2 * kb;
+    return kWsAlign + qb + 2 * kb;
 }
 
 rpx_status_t check_cache(const rpx_kv_cache_t* c, int32_t batch) {
@@ -75,7 +77,7 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.k_tok_stride = k_tok_stride;
     a.v_tok_stride = v_tok_stride;
     if (desc->dtype == RPX_F32) {
-        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        uint8_t* ws = static_cast<uint8_t*>(workspace) + kWsAlign;
         const size_t qb = align_up(static_cast<size_t>(total_tokens) * q_row * 2, kWsAlign);
         const size_t kb = align_up(static_cast<size_t>(total_tokens) * kv_row * 2, kWsAlign);
         auto* qh = reinterpret_cast<__nv_bfloat16_raw*>(ws);
@@ -98,6 +100,7 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.max_q_len = max_q_len;
     a.max_prefix_len = max_prefix_len;
     a.cache = cache;
+    a.item_counter = static_cast<uint32_t*>(workspace);
     a.append_cache = is_suffix && append_cache;
     a.out = out;
     a.out_f32 = desc->dtype == RPX_F32;

@@ -32,6 +32,7 @@ namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
 constexpr int kSlots = 5;
+constexpr int kItemRing = 4;  // work-item ids the producer may hand out ahead of the slowest warp
 constexpr int kChunks = kTileK / 32;  // 32-column TMEM loads per row and step
 constexpr int kWarpsPerTile = 4;
 constexpr int kProducerWarp = 2 * kWarpsPerTile, kMmaWarp = kProducerWarp + 1;
@@ -51,7 +52,12 @@ struct Ctl {
     uint64_t kv_empty[kSlots];
     uint64_t s_full[2];   // tensor core -> softmax: S_t(j) is in TMEM (and PV_t(j-1) has finished)
     uint64_t p_ready[2];  // softmax -> tensor core: P_t(j) is in TMEM, O_t rescaled if needed
-    uint64_t o_done[2];   // tensor core -> softmax: the last PV_t has finished
+    uint64_t o_done[2];   // tensor core -> softmax: the last PV_t of the work item has finished
+    uint64_t o_free[2];   // softmax -> tensor core: O_t of the finished item has been read out of TMEM
+    uint64_t q_empty;     // tensor core -> producer: the item's last Q K^T has finished, Q may be overwritten
+    uint64_t item_full[kItemRing];   // producer -> everyone: item_id[k] holds the next work item
+    uint64_t item_empty[kItemRing];  // everyone -> producer: item_id[k] has been read
+    int32_t item_id[kItemRing];
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -81,7 +87,9 @@ struct Params {
     __nv_bfloat16* v_cache;
     int32_t write_cache;          // store this call's K/V into the cache (prefix pass, chunked prefill)
     int32_t batch, num_q_heads, num_kv_heads, group;
-    int32_t n_pairs;              // query tile pairs per sequence the grid covers
+    int32_t n_pairs;              // query tile pairs per sequence the work list covers
+    int32_t n_items;              // n_pairs * batch * num_q_heads
+    uint32_t* next_item;          // device counter, zero before the launch: work items are handed out in order
     float scale_log2;
     void* out;
     int32_t out_f32;
@@ -94,34 +102,43 @@ __device__ __forceinline__ uint32_t swz_off(int r, int cc) {
     return static_cast<uint32_t>((cc >> 3) * (kTileK * 128) + r * 128 + (((cc & 7) ^ (r & 7)) << 4));
 }
 
+// One work item = two adjacent 128-row query tiles of one (sequence, query head).  Items are numbered
+// so that late query tiles (most keys, longest work) come first; CTAs take them in that order from a
+// device counter, so the longest items start first and the short ones fill the tail.
+struct Item {
+    int32_t pair, seq, head, kv_head, tok0, len_q, q0, len_p, n_prefix_tiles, n_tile0, n_kv;
+    bool active, active1;
+};
+
+__device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
+    Item it;
+    const int32_t per_pair = p.batch * p.num_q_heads;
+    it.pair = p.n_pairs - 1 - idx / per_pair;
+    const int32_t rem = idx % per_pair;
+    it.seq = rem / p.num_q_heads;
+    it.head = rem % p.num_q_heads;
+    it.kv_head = it.head / p.group;
+    it.tok0 = p.cu_seqlens[it.seq];
+    it.len_q = p.cu_seqlens[it.seq + 1] - it.tok0;
+    it.q0 = it.pair * 2 * kTileQ;
+    it.active = it.q0 < it.len_q;
+    it.len_p = (it.active && p.prefix_lens != nullptr) ? p.prefix_lens[it.seq] : 0;
+    it.active1 = it.q0 + kTileQ < it.len_q;
+    it.n_prefix_tiles = (it.len_p + kTileK - 1) / kTileK;
+    // key tiles seen by query tile t: n_tile0 + t.  (Scalars, not arrays: a small array indexed at
+    // run time lives in local memory, and with nearly all L1 carved out as shared memory every such
+    // load stalls the in-order warp for hundreds of cycles.)
+    it.n_tile0 = it.n_prefix_tiles + 2 * it.pair + 1;
+    it.n_kv = it.active1 ? it.n_tile0 + 1 : it.n_tile0;
+    return it;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
             const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
             const __grid_constant__ CUtensorMap tmap_vc, const Params p) {
     using L = Layout<D>;
-    // ---- which (pair, sequence, head) this CTA owns; late query tiles (most keys) launch first
-    const int32_t per_pair = p.batch * p.num_q_heads;
-    const int32_t pair = p.n_pairs - 1 - static_cast<int32_t>(blockIdx.x / per_pair);
-    const int32_t rem = static_cast<int32_t>(blockIdx.x % per_pair);
-    const int32_t seq = rem / p.num_q_heads;
-    const int32_t head = rem % p.num_q_heads;
-    const int32_t kv_head = head / p.group;
-    const int32_t tok0 = p.cu_seqlens[seq];
-    const int32_t len_q = p.cu_seqlens[seq + 1] - tok0;
-    const int32_t q0 = pair * 2 * kTileQ;
-    // A sequence longer than the caller's bound would leave rows the grid never reaches: report it.
-    if (pair == 0 && threadIdx.x == 0 && head == 0 && len_q > p.n_pairs * 2 * kTileQ && p.status != nullptr)
-        atomicCAS(p.status, 0, RPX_ERR_DEVICE_DATA);
-    if (q0 >= len_q) return;  // uniform for the whole CTA, before any barrier or allocation
-    const int32_t len_p = p.prefix_lens != nullptr ? p.prefix_lens[seq] : 0;
-    const bool active1 = q0 + kTileQ < len_q;
-    const int32_t n_prefix_tiles = (len_p + kTileK - 1) / kTileK;
-    // key tiles seen by query tile t: n_tile0 + t.  (Scalars, not arrays: a small array indexed at
-    // run time lives in local memory, and with nearly all L1 carved out as shared memory every such
-    // load stalls the in-order warp for hundreds of cycles.)
-    const int32_t n_tile0 = n_prefix_tiles + 2 * pair + 1;
-    const int32_t n_kv = active1 ? n_tile0 + 1 : n_tile0;
     // Rows that see only a handful of keys (the first rows of a sequence with little or no cached
     // prefix) get no averaging over keys, so the 2^-9 rounding of each bf16 probability shows up in
     // O at full size (up to 2^-9 * |v|) and, stacked on the bf16 rounding of O itself, can pass 1e-2.
@@ -129,6 +146,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     // of a sequence with at most one tile of cached prefix).  For it the probabilities are kept as
     // two bf16 terms, P = P_hi + P_lo, with P_lo in the unused upper half of S_t's columns and a
     // second PV MMA: exact to 2^-17 at the cost of at most four extra MMA groups per sequence and head.
+    //
+    // The CTA is persistent: it takes work items until the list is empty.  The producer warp draws the
+    // item numbers from the device counter and hands them to the other warps through a small ring, so
+    // it can fetch the next item's Q and first K tiles while the softmax warps still write the current
+    // item's output; barrier parities run on counters that carry over from item to item.
 
     extern __shared__ __align__(1024) uint8_t smem[];
     if ((smem_u32(smem) & 1023u) != 0u) {  // swizzled tiles need 1024-byte alignment; never expected
@@ -150,6 +172,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             mbar_init(&ctl->s_full[t], 1);
             mbar_init(&ctl->p_ready[t], kWarpsPerTile);  // one arrival per softmax warp
             mbar_init(&ctl->o_done[t], 1);
+        }
+        for (int t = 0; t < 2; ++t) mbar_init(&ctl->o_free[t], kWarpsPerTile);
+        mbar_init(&ctl->q_empty, 1);
+        for (int k = 0; k < kItemRing; ++k) {
+            mbar_init(&ctl->item_full[k], 1);
+            mbar_init(&ctl->item_empty[k], 2 * kWarpsPerTile + 1);  // every softmax warp and the issuer
         }
         mbar_init(&ctl->drain, 1);
         ctl->abort_flag = 0;
@@ -174,6 +202,43 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             tma_prefetch_desc(&tmap_q);
             tma_prefetch_desc(&tmap_k);
             tma_prefetch_desc(&tmap_v);
+        }
+        uint32_t n_loaded = 0;  // K/V tiles loaded so far (ring position)
+        uint32_t n_fetched = 0; // work items drawn so far (item ring position)
+        uint32_t n_active = 0;  // of those, items with any rows (parity of the Q barriers)
+        for (;;) {
+            // ---- draw the next work item and hand its number to the other warps
+            const uint32_t ring = n_fetched % kItemRing;
+            if (!mbar_wait(&ctl->item_empty[ring], ((n_fetched / kItemRing) & 1u) ^ 1u, abort_flag)) {
+                ok = false;
+                break;
+            }
+            int32_t idx = 0;
+            if (lane == 0) {
+                idx = static_cast<int32_t>(atomicAdd(p.next_item, 1u));
+                if (idx >= p.n_items) idx = -1;
+                ctl->item_id[ring] = idx;
+                mbar_arrive(&ctl->item_full[ring]);
+            }
+            idx = __shfl_sync(0xffffffffu, idx, 0);
+            ++n_fetched;
+            if (idx < 0) break;
+            const Item it = decode_item(p, idx);
+            // A sequence longer than the caller's bound would leave rows the work list never reaches: report it.
+            if (it.pair == 0 && it.head == 0 && lane == 0 && it.len_q > p.n_pairs * 2 * kTileQ) ctl->data_error = 1;
+            if (!it.active) continue;
+            const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
+            const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const bool active1 = it.active1;
+            (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
+            // ---- Q of this item, once the previous item's last Q K^T has let go of the buffer
+            if (n_active > 0 && !mbar_wait(&ctl->q_empty, (n_active - 1) & 1u, abort_flag)) {
+                ok = false;
+                break;
+            }
+            if (lane == 0) {
             mbar_arrive_expect_tx(&ctl->q_full, (active1 ? 2 : 1) * L::kQBytes);
             for (int t = 0; t < (active1 ? 2 : 1); ++t)
                 for (int hf = 0; hf < L::kHalves; ++hf)
@@ -186,7 +251,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         if (p.write_cache != 0 && !page_aligned && lane == 0) ctl->data_error = 1;
         const bool owns_cache_write = p.write_cache != 0 && page_aligned && (head % p.group) == 0;
         const int32_t write_page0 = len_p / kPage;  // first page of this call's own tokens
-        uint32_t n_loaded = 0;
         // Block id of page `lane` of cached tile jt (lanes 0..7; 0 where the prefix has no such page).
         // Read one tile ahead, so the table's global-memory latency is off the ring's critical path.
         auto read_block_ids = [&](int32_t jt) -> int32_t {
@@ -306,13 +370,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 }
             }
         }
+            ++n_active;
+            if (!ok) break;
+        }
         if (lane == 0) tma_store_wait_all();
         if (!ok) {
             // abort: give copies already in flight a moment to land before smem is released
             const uint32_t first = n_loaded > kSlots ? n_loaded - kSlots : 0u;
             for (uint32_t i = first; i < n_loaded; ++i)
                 mbar_wait(&ctl->kv_full[i % kSlots], (i / kSlots) & 1u, &ctl->drain_flag, kDrainLimitCycles);
-            mbar_wait(&ctl->q_full, 0, &ctl->drain_flag, kDrainLimitCycles);
+            if (n_active > 0) mbar_wait(&ctl->q_full, (n_active - 1) & 1u, &ctl->drain_flag, kDrainLimitCycles);
         }
     } else if (warp == kMmaWarp) {
         // =========================================================== tcgen05 issuer (one thread)
@@ -327,6 +394,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             const uint64_t q_desc0 = make_smem_desc_sw128(q_addr, 16, 1024);
             const uint64_t k_desc0 = make_smem_desc_sw128(kv_addr, 16, 1024);             // K tile: K-major
             const uint64_t v_desc0 = make_smem_desc_sw128(kv_addr, L::kHalfBytes, 1024);  // V tile: MN-major
+            uint32_t n_seen = 0;              // work items read from the item ring
+            uint32_t n_active = 0;            // items with rows so far = items in which tile 0 took part
+            uint32_t items1 = 0;              // items in which tile 1 took part
+            uint32_t cnt0 = 0, cnt1 = 0;      // key steps tile 0 / tile 1 have been through (barrier parity)
+            uint32_t kv_base = 0;             // K/V tiles consumed before this item
+            for (;;) {
+            const uint32_t ring = n_seen % kItemRing;
+            if (!mbar_wait(&ctl->item_full[ring], (n_seen / kItemRing) & 1u, abort_flag)) {
+                ok = false;
+                break;
+            }
+            const int32_t idx = *reinterpret_cast<volatile int32_t*>(&ctl->item_id[ring]);
+            mbar_arrive(&ctl->item_empty[ring]);
+            ++n_seen;
+            if (idx < 0) break;
+            const Item it = decode_item(p, idx);
+            if (!it.active) continue;
+            const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
+            const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const bool active1 = it.active1;
+            (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
             auto issue_qk = [&](int t, uint32_t k_slot) {
                 const uint64_t kd = k_desc0 + static_cast<uint64_t>(k_slot * (L::kKvBytes >> 4));
                 const uint64_t qd = q_desc0 + static_cast<uint64_t>(t * (L::kQBytes >> 4));
@@ -342,23 +432,33 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128 + 64, vd, idesc_pv, 1u);
             };
 
-            ok = mbar_wait(&ctl->q_full, 0, abort_flag);
-            if (ok) ok = mbar_wait(&ctl->kv_full[0], 0, abort_flag);  // K_0 is load 0
+            ok = mbar_wait(&ctl->q_full, n_active & 1u, abort_flag);
+            const uint32_t k0_slot = kv_base % kSlots;  // K_0 is the item's first load
+            if (ok) ok = mbar_wait(&ctl->kv_full[k0_slot], (kv_base / kSlots) & 1u, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
-                issue_qk(0, 0);
-                if (active1) issue_qk(1, 0);
-                umma_commit(&ctl->kv_empty[0]);
+                issue_qk(0, k0_slot);
+                if (active1) issue_qk(1, k0_slot);
+                umma_commit(&ctl->kv_empty[k0_slot]);
+                if (n_kv == 1) umma_commit(&ctl->q_empty);  // no further Q K^T in this item
             }
             for (int32_t j = 0; ok && j < n_kv; ++j) {
-                const uint32_t v_idx = 2 * j + 1, kn_idx = 2 * j + 2;
+                const uint32_t v_idx = kv_base + 2 * j + 1, kn_idx = kv_base + 2 * j + 2;
                 const uint32_t v_slot = v_idx % kSlots, kn_slot = kn_idx % kSlots;
                 bool have_v = false, have_kn = false;
                 for (int t = 0; t < 2 && ok; ++t) {
                     if ((t == 1 && !active1) || j >= n_tile0 + t) continue;
-                    if (!mbar_wait(&ctl->p_ready[t], j & 1, abort_flag)) {
+                    if (!mbar_wait(&ctl->p_ready[t], ((t ? cnt1 : cnt0) + j) & 1u, abort_flag)) {
                         ok = false;
                         break;
+                    }
+                    if (j == 0) {
+                        // the first PV of an item overwrites O_t: the previous item's output must have left TMEM
+                        const uint32_t before = t ? items1 : n_active;
+                        if (before > 0 && !mbar_wait(&ctl->o_free[t], (before - 1) & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
                     }
                     if (!have_v) {
                         if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag)) {
@@ -386,6 +486,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 if (!ok) break;
                 umma_commit(&ctl->kv_empty[v_slot]);
                 if (have_kn) umma_commit(&ctl->kv_empty[kn_slot]);
+                if (j == n_kv - 2) umma_commit(&ctl->q_empty);  // the item's last Q K^T went out in this step
+            }
+            if (!ok) break;
+            kv_base += 2u * static_cast<uint32_t>(n_kv);
+            cnt0 += static_cast<uint32_t>(n_tile0);
+            if (active1) {
+                cnt1 += static_cast<uint32_t>(n_tile0) + 1u;
+                ++items1;
+            }
+            ++n_active;
             }
             if (!ok) {
                 umma_commit(&ctl->drain);
@@ -396,7 +506,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     } else {
         // =========================================================== softmax warps
         const int t = warp / kWarpsPerTile;
-        if (t == 0 || active1) {
+        uint32_t n_seen = 0;  // work items read from the item ring
+        uint32_t cnt = 0;     // key steps this tile has been through (barrier parity)
+        uint32_t items_t = 0; // items this tile took part in
+        bool ok = true;
+        while (ok) {
+            const uint32_t ring = n_seen % kItemRing;
+            if (!mbar_wait(&ctl->item_full[ring], (n_seen / kItemRing) & 1u, abort_flag)) break;
+            const int32_t idx = *reinterpret_cast<volatile int32_t*>(&ctl->item_id[ring]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->item_empty[ring]);
+            ++n_seen;
+            if (idx < 0) break;
+            const Item it = decode_item(p, idx);
+            if (!it.active || (t == 1 && !it.active1)) continue;
+            const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
+            const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const bool active1 = it.active1;
+            (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
             const uint32_t quarter = warp & 3;
             const int32_t row = quarter * 32 + lane;
             const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
@@ -405,13 +534,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             const uint32_t my_s = tmem_base + t * 128 + lane_addr;        // this thread's lane of S_t / P_t
             const uint32_t my_o = tmem_base + 256 + t * 128 + lane_addr;  // and of O_t
             float run_max = -CUDART_INF_F, run_sum = 0.f;
-            bool ok = true;
             // The whole step loop is instantiated twice, so the common (kSplit = false) instance is
             // scheduled and register-allocated exactly as if the two-term variant did not exist.
             auto run_steps = [&](auto split_tag) {
               constexpr bool kSplit = decltype(split_tag)::value;
               for (int32_t j = 0; j < my_tiles; ++j) {
-                if (!mbar_wait(&ctl->s_full[t], j & 1, abort_flag)) {
+                if (!mbar_wait(&ctl->s_full[t], (cnt + j) & 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
@@ -523,7 +651,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             else
                 run_steps(std::false_type{});
             // ---- epilogue: O / l -> global, LSE
-            if (ok) ok = mbar_wait(&ctl->o_done[t], 0, abort_flag);
+            cnt += static_cast<uint32_t>(my_tiles);
+            if (ok) ok = mbar_wait(&ctl->o_done[t], items_t & 1u, abort_flag);
+            ++items_t;
             if (ok) {
                 tc_fence_after_sync();
                 const bool row_valid = q_local < len_q;
@@ -534,6 +664,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     uint32_t r[32];
                     tmem_ld32(my_o + c * 32, r);
                     tmem_ld_wait();
+                    if (c == D / 32 - 1) {  // O_t is out of TMEM: the next item's first PV may overwrite it
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&ctl->o_free[t]);
+                    }
                     if (row_valid) {
                         if (p.out_f32) {
                             float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + out_row + c * 32);
@@ -622,9 +757,16 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.out_f32 = a.out_f32 ? 1 : 0;
     p.lse = a.lse;
     p.status = a.device_status;
-    const int64_t grid = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
-    if (grid <= 0) return RPX_OK;
-    if (grid > INT32_MAX) return RPX_ERR_SHAPE;
+    const int64_t n_items = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
+    if (n_items <= 0) return RPX_OK;
+    if (n_items > INT32_MAX - 65536) return RPX_ERR_SHAPE;  // the counter runs past n_items by one draw per CTA
+    if (a.item_counter == nullptr) return RPX_ERR_WORKSPACE;
+    p.n_items = static_cast<int32_t>(n_items);
+    p.next_item = a.item_counter;
+    const int sms = sm_count();
+    if (sms <= 0) return RPX_ERR_CUDA;
+    const int64_t grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM
+    if (cudaMemsetAsync(a.item_counter, 0, sizeof(uint32_t), a.stream) != cudaSuccess) return RPX_ERR_CUDA;
     if (cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(L::kSmemBytes)) != cudaSuccess)
         return RPX_ERR_CUDA;

@@ -38,6 +38,7 @@ struct AttnArgs {
     int32_t max_q_len, max_prefix_len;
     const rpx_kv_cache_t* cache;       // prefix pass: written (nullable); suffix pass: read
     bool append_cache = false;         // chunked prefill: read the earlier chunks AND append this one
+    uint32_t* item_counter = nullptr;  // 4 bytes of workspace: the kernel's work-item counter (zeroed by the launcher)
     void* out;
     bool out_f32;
     float* lse;

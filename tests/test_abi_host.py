@@ -51,10 +51,12 @@ def test_sm_budget_is_host_state_with_validation(lib):
 
 
 def test_workspace_arithmetic(lib):
-    assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 32768) == 0
+    # every attention call keeps its work-item counter in the first 256 bytes; fp32 calls add bf16 copies of q, k, v
+    assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 32768) == 256
+    assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 0) == 0
     need = B.prefix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 256)
-    assert need == 256 * 4 * 64 * 2 + 2 * 256 * 2 * 64 * 2
-    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 32 * 8 * 64 * 2
+    assert need == 256 + 256 * 4 * 64 * 2 + 2 * 256 * 2 * 64 * 2
+    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 256 + 32 * 8 * 64 * 2
     # 152064 columns = 594 tiles of 256; one float4 per (chunk, row): 38 chunks of 16 tiles up to 191 row
     # tiles of 128 rows, 75 chunks of 8 tiles from 192 row tiles on
     assert B.token_logprobs_workspace_bytes(12800, 3584, 152064, B.RPX_BF16) == 38 * 12800 * 16

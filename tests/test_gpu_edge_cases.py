@@ -43,8 +43,9 @@ def test_empty_batches_are_no_ops_on_the_device(cuda_device):
     q = torch.zeros((8, 4, 128), dtype=torch.bfloat16, device=dev)
     kv = torch.zeros((8, 2, 128), dtype=torch.bfloat16, device=dev)
     # three sequences of length zero inside a non-empty allocation: every CTA exits at once
+    ws = torch.empty(256, dtype=torch.uint8, device=dev)  # the kernel's work-item counter lives here
     rc = lib.rpx_prefix_attn(ctypes.byref(desc), q.data_ptr(), kv.data_ptr(), kv.data_ptr(), 512, 256, 256, cu.data_ptr(),
-                             3, 8, 256, None, out.data_ptr(), None, None, 0, None, None)
+                             3, 8, 256, None, out.data_ptr(), None, ws.data_ptr(), 256, None, None)
     torch.cuda.synchronize()
     assert rc == 0 and bool((out == 7.0).all())
     assert lib.rpx_prefix_attn(ctypes.byref(desc), None, None, None, 512, 256, 256, None, 0, 0, 0, None, None, None, None,
