@@ -1,14 +1,15 @@
 // Varlen causal GQA flash attention for sm_100a, shared by the prefix pass (which also writes the
 // paged boundary-KV cache) and the suffix pass (which reads it back through the block table).
 //
-// One CTA owns two adjacent 128-row query tiles of one (sequence, query head) and walks the key
-// tiles (128 keys) that those rows may see: first the cached prefix tiles (suffix pass only,
+// A work item is two adjacent 128-row query tiles of one (sequence, query head); the kernel is
+// persistent (one CTA per SM) and its CTAs draw items, longest first, from a device counter.  For an
+// item the CTA walks the key tiles (128 keys) that those rows may see: first the cached prefix tiles (suffix pass only,
 // unmasked except the last partial one), then the self tiles up to each query tile's diagonal.
 //   warps 0-3 : softmax of query tile 0: thread = one row = one TMEM lane, all 128 scores of the
 //               row in registers (two threads per row were tried: the extra exchange of the row
 //               maximum cost more than the shorter dependency chains gained)
 //   warps 4-7 : softmax of query tile 1
-//   warp  8   : TMA producer (Q once; K/V through a 5-slot ring; paged tiles = one TMA box per
+//   warp  8   : TMA producer (Q once; K/V through a 4-slot ring; paged tiles = one TMA box per
 //               16-token page); it also stores the diagonal K/V tiles into the paged cache
 //   warp  9   : TMEM owner and tcgen05 issuer:  S_t = Q_t K^T  (smem x smem -> TMEM),
 //               O_t += P_t V  (P_t = bf16 probabilities written back into the first 64 columns
@@ -31,7 +32,7 @@ namespace rpx {
 namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
-constexpr int kSlots = 5;
+constexpr int kSlots = 4;  // K/V tiles in flight (two key steps); a fifth slot measured no faster
 constexpr int kItemRing = 4;  // work-item ids the producer may hand out ahead of the slowest warp
 constexpr int kChunks = kTileK / 32;  // 32-column TMEM loads per row and step
 constexpr int kWarpsPerTile = 4;
@@ -57,7 +58,7 @@ struct Ctl {
     uint64_t q_empty;     // tensor core -> producer: the item's last Q K^T has finished, Q may be overwritten
     uint64_t item_full[kItemRing];   // producer -> everyone: item_id[k] holds the next work item
     uint64_t item_empty[kItemRing];  // everyone -> producer: item_id[k] has been read
-    int32_t item_id[kItemRing];
+    int4 item_rec[kItemRing];        // (item number or -1, first token, query length, cached prefix length)
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -110,19 +111,35 @@ struct Item {
     bool active, active1;
 };
 
-__device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
+// The lengths come from device memory once per item (the producer's lane 0 reads them, a tile ahead of
+// everyone else, and passes them on through shared memory); the rest is arithmetic on the item number.
+__device__ __forceinline__ int4 fetch_item(const Params& p, int32_t idx) {
+    const int32_t seq = (idx % (p.batch * p.num_q_heads)) / p.num_q_heads;
+    const int32_t tok0 = __ldg(p.cu_seqlens + seq);
+    const int32_t len_q = __ldg(p.cu_seqlens + seq + 1) - tok0;
+    const int32_t len_p = p.prefix_lens != nullptr ? __ldg(p.prefix_lens + seq) : 0;
+    return make_int4(idx, tok0, len_q, len_p);
+}
+
+__device__ __forceinline__ int4 read_item_rec(const int4* rec) {
+    const volatile int32_t* w = reinterpret_cast<const volatile int32_t*>(rec);
+    return make_int4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ Item decode_item(const Params& p, int4 rec) {
     Item it;
+    const int32_t idx = rec.x;
     const int32_t per_pair = p.batch * p.num_q_heads;
     it.pair = p.n_pairs - 1 - idx / per_pair;
     const int32_t rem = idx % per_pair;
     it.seq = rem / p.num_q_heads;
     it.head = rem % p.num_q_heads;
     it.kv_head = it.head / p.group;
-    it.tok0 = p.cu_seqlens[it.seq];
-    it.len_q = p.cu_seqlens[it.seq + 1] - it.tok0;
+    it.tok0 = rec.y;
+    it.len_q = rec.z;
     it.q0 = it.pair * 2 * kTileQ;
     it.active = it.q0 < it.len_q;
-    it.len_p = (it.active && p.prefix_lens != nullptr) ? p.prefix_lens[it.seq] : 0;
+    it.len_p = it.active ? rec.w : 0;
     it.active1 = it.q0 + kTileQ < it.len_q;
     it.n_prefix_tiles = (it.len_p + kTileK - 1) / kTileK;
     // key tiles seen by query tile t: n_tile0 + t.  (Scalars, not arrays: a small array indexed at
@@ -213,17 +230,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 ok = false;
                 break;
             }
-            int32_t idx = 0;
+            int4 rec = make_int4(-1, 0, 0, 0);
             if (lane == 0) {
-                idx = static_cast<int32_t>(atomicAdd(p.next_item, 1u));
-                if (idx >= p.n_items) idx = -1;
-                ctl->item_id[ring] = idx;
+                const int32_t idx = static_cast<int32_t>(atomicAdd(p.next_item, 1u));
+                if (idx < p.n_items) rec = fetch_item(p, idx);
+                ctl->item_rec[ring] = rec;
                 mbar_arrive(&ctl->item_full[ring]);
             }
-            idx = __shfl_sync(0xffffffffu, idx, 0);
+            rec.x = __shfl_sync(0xffffffffu, rec.x, 0);
+            rec.y = __shfl_sync(0xffffffffu, rec.y, 0);
+            rec.z = __shfl_sync(0xffffffffu, rec.z, 0);
+            rec.w = __shfl_sync(0xffffffffu, rec.w, 0);
             ++n_fetched;
-            if (idx < 0) break;
-            const Item it = decode_item(p, idx);
+            if (rec.x < 0) break;
+            const Item it = decode_item(p, rec);
             // A sequence longer than the caller's bound would leave rows the work list never reaches: report it.
             if (it.pair == 0 && it.head == 0 && lane == 0 && it.len_q > p.n_pairs * 2 * kTileQ) ctl->data_error = 1;
             if (!it.active) continue;
@@ -405,11 +425,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 ok = false;
                 break;
             }
-            const int32_t idx = *reinterpret_cast<volatile int32_t*>(&ctl->item_id[ring]);
+            const int4 rec = read_item_rec(&ctl->item_rec[ring]);
             mbar_arrive(&ctl->item_empty[ring]);
             ++n_seen;
-            if (idx < 0) break;
-            const Item it = decode_item(p, idx);
+            if (rec.x < 0) break;
+            const Item it = decode_item(p, rec);
             if (!it.active) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
@@ -513,12 +533,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         while (ok) {
             const uint32_t ring = n_seen % kItemRing;
             if (!mbar_wait(&ctl->item_full[ring], (n_seen / kItemRing) & 1u, abort_flag)) break;
-            const int32_t idx = *reinterpret_cast<volatile int32_t*>(&ctl->item_id[ring]);
+            const int4 rec = read_item_rec(&ctl->item_rec[ring]);
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->item_empty[ring]);
             ++n_seen;
-            if (idx < 0) break;
-            const Item it = decode_item(p, idx);
+            if (rec.x < 0) break;
+            const Item it = decode_item(p, rec);
             if (!it.active || (t == 1 && !it.active1)) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
@@ -659,36 +679,62 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const bool row_valid = q_local < len_q;
                 const float inv = 1.f / run_sum;
                 const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
-#pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(my_o + c * 32, r);
-                    tmem_ld_wait();
-                    if (c == D / 32 - 1) {  // O_t is out of TMEM: the next item's first PV may overwrite it
+                // two chunks of 32 columns in flight: the next chunk's TMEM load runs under this chunk's stores
+                uint32_t ra[32], rb[32];
+                // A warp's store instruction touches 32 rows, so its cost is the number of 32-byte sectors
+                // it writes: 32-byte stores (one full sector per row and instruction) halve the count
+                // against 16-byte ones.  They need the output base on a 32-byte boundary.
+                const bool wide = (reinterpret_cast<uintptr_t>(p.out) & 31u) == 0u;
+                auto store_chunk = [&](const uint32_t (&r)[32], int c) {
+                    if (!row_valid) return;
+                    if (p.out_f32) {
+                        float* dst = static_cast<float*>(p.out) + out_row + c * 32;
+                        uint32_t w[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(r[i]) * inv);
+                        if (wide) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                st_global_v8(dst + 8 * i, w[8 * i], w[8 * i + 1], w[8 * i + 2], w[8 * i + 3], w[8 * i + 4],
+                                             w[8 * i + 5], w[8 * i + 6], w[8 * i + 7]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                        }
+                    } else {
+                        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + out_row + c * 32;
+                        uint32_t w[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            w[i] = pack_bf16x2(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
+                        if (wide) {
+                            st_global_v8(dst, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                            st_global_v8(dst + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                        }
+                    }
+                };
+                tmem_ld32(my_o, ra);
+#pragma unroll
+                for (int c = 0; c < D / 32; c += 2) {
+                    tmem_ld32(my_o + (c + 1) * 32, rb);
+                    tmem_ld_wait();  // both loads: ra and rb are in registers
+                    if (c + 2 >= D / 32) {  // O_t is out of TMEM: the next item's first PV may overwrite it
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&ctl->o_free[t]);
+                    } else {
+                        store_chunk(ra, c);
+                        tmem_ld32(my_o + (c + 2) * 32, ra);
+                        store_chunk(rb, c + 1);
+                        continue;
                     }
-                    if (row_valid) {
-                        if (p.out_f32) {
-                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + out_row + c * 32);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
-                                                     __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
-                        } else {
-                            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + out_row + c * 32);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int u = 0; u < 4; ++u)
-                                    w[u] = pack_bf16x2(__uint_as_float(r[8 * i + 2 * u]) * inv,
-                                                       __uint_as_float(r[8 * i + 2 * u + 1]) * inv);
-                                dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
-                    }
+                    store_chunk(ra, c);
+                    store_chunk(rb, c + 1);
                 }
                 if (row_valid && p.lse != nullptr)
                     p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
