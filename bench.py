@@ -42,7 +42,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the LM-head partial kernel on the
 # benchmark's prompt-row launch (32768 x 152064 x 3584), from a one-pass ncu capture of this very
 # command; summary in profiles/lm_head_partial_kernel__slice_8192x32768x3584.md.  Other configs: None.
-LM_HEAD_TRAFFIC_BYTES = {"C2": 11.40e9 + 24.0e6}
+LM_HEAD_TRAFFIC_BYTES = {"C2": 13.291e9 + 43.8e6}
 
 
 def load_peaks():
