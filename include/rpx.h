@@ -249,12 +249,11 @@ RPX_API rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* de
 /*
  * SM budget for co-running (Section 3.1, Eq. 1).  The overlap model charges the decode side a
  * slowdown Delta_D for sharing the GPU with prefix work; how large it is depends on how much of
- * the GPU the prefix kernels leave free.  The LM-head kernel is persistent (one CTA per SM, all
- * shared memory of the SM), so left alone it leaves nothing.  rpx_set_sm_budget(n) caps its grid
- * at n CTAs for every later rpx_token_logprobs* call of this process (all devices, all streams);
+ * the GPU the prefix kernels leave free.  The LM-head and attention kernels are persistent (one
+ * CTA per SM, all shared memory of the SM), so left alone they leave nothing.  rpx_set_sm_budget(n)
+ * caps their grids at n CTAs for every later call of this process (all devices, all streams);
  * 0 removes the cap, n < 0 returns RPX_ERR_SHAPE and changes nothing.  Results do not depend on
- * the budget bit for bit.  The attention kernels are not persistent (one short CTA per work item)
- * and are not capped.  Host-only state: no CUDA call, no allocation, nothing set on the GPU.
+ * the budget bit for bit.  Host-only state: no CUDA call, no allocation, nothing set on the GPU.
  */
 RPX_API rpx_status_t rpx_set_sm_budget(int32_t sms);
 RPX_API int32_t rpx_get_sm_budget(void);

@@ -211,7 +211,7 @@ def selftest_bounded_wait(limit_cycles: int, device_status, stream=None) -> None
 
 
 def set_sm_budget(sms: int) -> None:
-    """rpx_set_sm_budget: cap the persistent LM-head grid at ``sms`` CTAs (0 = no cap), process-wide."""
+    """rpx_set_sm_budget: cap the persistent kernels' grids at ``sms`` CTAs (0 = no cap), process-wide."""
     rc = load_library().rpx_set_sm_budget(int(sms))
     if rc != 0:
         raise RpxError(rc, "rpx_set_sm_budget")

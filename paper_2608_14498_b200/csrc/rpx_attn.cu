@@ -809,8 +809,9 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     if (a.item_counter == nullptr) return RPX_ERR_WORKSPACE;
     p.n_items = static_cast<int32_t>(n_items);
     p.next_item = a.item_counter;
-    const int sms = sm_count();
+    int sms = sm_count();
     if (sms <= 0) return RPX_ERR_CUDA;
+    if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;  // leave the rest to a co-runner
     const int64_t grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM
     if (cudaMemsetAsync(a.item_counter, 0, sizeof(uint32_t), a.stream) != cudaSuccess) return RPX_ERR_CUDA;
     if (cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -142,6 +142,20 @@ def test_prefix_without_cache_and_explicit_scale(cuda_device):
     assert err <= TOL
 
 
+def test_sm_budget_changes_no_bit_of_the_attention_outputs(cuda_device):
+    cfg = wk.Config("t", "bf16", 3, 4, 2, 128, 64, 64, ("list", [600, 333, 48]), ("list", [100, 20, 260]))
+    wl = wk.make_workload(cfg, seed=15, lm=False)
+    _, _, kc1, vc1, (p1, s1) = run_split(wl, cuda_device)
+    try:
+        for budget in (1, 5, 147):
+            rpx.set_sm_budget(budget)
+            _, _, kc2, vc2, (p2, s2) = run_split(wl, cuda_device)
+            assert torch.equal(p1, p2) and torch.equal(s1, s2)
+            assert np.array_equal(kc1, kc2) and np.array_equal(vc1, vc2)
+    finally:
+        rpx.set_sm_budget(0)
+
+
 @pytest.mark.parametrize("growth", [40.0, 400.0])
 def test_scores_that_keep_growing_force_the_running_maximum_to_move(cuda_device, growth):
     """Key norms grow along the sequence, so every 128-key tile raises the row maximum by tens
