@@ -131,9 +131,9 @@ class ScoringSession:
         """Pinned host batch in, log-probs out into the pinned ``lp_*_host`` tensors.
 
         Host->device copies run on a copy stream in the order the kernels need them and each
-        kernel waits only for its own inputs: the prompt rows of the LM head (the longest kernel)
-        are cut into ``lm_slices`` row slices so that scoring starts after the first slice has
-        landed and the remaining copies hide behind it.  Kernels and the device->host copy of the
+        kernel waits only for its own inputs: the rows of the LM head (the longest kernels) are cut
+        into row slices (``lm_slices`` for the prompt rows, the response rows in proportion) so that
+        scoring starts after the first slice has landed and the remaining copies hide behind it.  Kernels and the device->host copy of the
         results are enqueued on the current stream; the caller synchronises.  Two staging sets
         alternate, so back-to-back calls overlap one pass's uploads with the previous pass's kernels."""
         t = self.torch
@@ -164,49 +164,68 @@ class ScoringSession:
                 ev.record(copy)
             return ev
 
-        n_p = hb.hidden_p.shape[0]
-        # a short first slice (1/16 of the rows) gets the first kernel going early; the rest is cut evenly
-        first = min(n_p, -(-(n_p // 16) // 128) * 128) if lm_slices > 1 else n_p
-        rest = max(lm_slices - 1, 1)
-        bounds = [0] + [first + (n_p - first) * i // rest for i in range(rest + 1)] if n_p > 0 else [0, 0]
-        bounds = sorted(set(bounds)) if n_p > 0 else bounds
-        ev_ids = upload([(d.ids_p, hb.ids_p)])
-        ev_slices = [upload([(d.hidden_p[a:b], hb.hidden_p[a:b])]) for a, b in zip(bounds[:-1], bounds[1:])]
+        n_p, n_s = hb.hidden_p.shape[0], hb.hidden_s.shape[0]
+
+        def cut(n, parts, short_first):
+            """Row bounds of ``parts`` slices of n rows; optionally a short first slice (1/16 of the rows,
+            a multiple of 128) so the first kernel can start early."""
+            if n <= 0:
+                return [0, 0]
+            first = min(n, -(-(n // 16) // 128) * 128) if (short_first and parts > 1) else 0
+            rest = max(parts - (1 if first else 0), 1)
+            return sorted(set([0] + [first + (n - first) * i // rest for i in range(rest + 1)]))
+
+        bounds_p = cut(n_p, lm_slices, True)
+        # response rows: slices of about the same size as the prompt-row slices, at most 8
+        bounds_s = cut(n_s, max(1, min(8, round(lm_slices * n_s / max(n_p, 1)), n_s // 4096)), False)
+        # Upload order = the order the kernels below consume their inputs.  The response rows of the LM
+        # head run before the suffix attention (the two are independent), so that the large q/k/v of the
+        # responses, needed last, also arrive last.
+        ev_ids = upload([(d.ids_p, hb.ids_p), (d.ids_s, hb.ids_s)])
+        ev_p = [upload([(d.hidden_p[a:b], hb.hidden_p[a:b])]) for a, b in zip(bounds_p[:-1], bounds_p[1:])]
         ev_prefix = upload([(d.q_p, hb.q_p), (d.k_p, hb.k_p), (d.v_p, hb.v_p), (d.cu_prefix, hb.cu_prefix),
                             (d.block_table, hb.block_table)])
+        ev_s = [upload([(d.hidden_s[a:b], hb.hidden_s[a:b])]) for a, b in zip(bounds_s[:-1], bounds_s[1:])]
         ev_suffix = upload([(d.q_s, hb.q_s), (d.k_s, hb.k_s), (d.v_s, hb.v_s), (d.cu_suffix, hb.cu_suffix),
-                            (d.prefix_lens, hb.prefix_lens), (d.hidden_s, hb.hidden_s), (d.ids_s, hb.ids_s)])
+                            (d.prefix_lens, hb.prefix_lens)])
 
         cache = (self.k_cache, self.v_cache, d.block_table)
         code = B._dtype_code(d.hidden_p)
         vocab, hdim = self.w_vocab.shape
         lp_p = self._buf("lp_p", (n_p,), t.float32)
-        lp_s = self._buf("lp_s", (hb.hidden_s.shape[0],), t.float32)
+        lp_s = self._buf("lp_s", (n_s,), t.float32)
         o_p = self._buf("o_p", d.q_p.shape, d.q_p.dtype)
         o_s = self._buf("o_s", d.q_s.shape, d.q_s.dtype)
-        lm_calls = [b - a for a, b in zip(bounds[:-1], bounds[1:])] + [hb.hidden_s.shape[0]]
+        lm_calls = [b - a for a, b in zip(bounds_p[:-1], bounds_p[1:])] + [b - a for a, b in zip(bounds_s[:-1], bounds_s[1:])]
         lm_ws = self._workspace("lm", max(B.token_logprobs_workspace_bytes(n, hdim, vocab, code) for n in lm_calls))
         attn_ws = self._workspace("attn", max(
             B.prefix_attn_workspace_bytes(d.q_p.shape[1], d.k_p.shape[1], d.q_p.shape[2], B._dtype_code(d.q_p), d.q_p.shape[0]),
             B.suffix_attn_workspace_bytes(d.q_s.shape[1], d.k_s.shape[1], d.q_s.shape[2], B._dtype_code(d.q_s), d.q_s.shape[0])))
+        n_lm = 0
         main.wait_event(ev_ids)
-        for (a, b), ev in zip(zip(bounds[:-1], bounds[1:]), ev_slices):
+        for (a, b), ev in zip(zip(bounds_p[:-1], bounds_p[1:]), ev_p):
             main.wait_event(ev)
             if b > a:
                 B.token_logprobs(d.hidden_p[a:b], self.w_vocab, d.ids_p[a:b], logprobs=lp_p[a:b], workspace=lm_ws,
                                  device_status=self.status)
+                n_lm += 1
         main.wait_event(ev_prefix)
         B.prefix_attn(d.q_p, d.k_p, d.v_p, d.cu_prefix, d.max_prefix_len, cache=cache, out=o_p, workspace=attn_ws,
                       device_status=self.status)
+        for (a, b), ev in zip(zip(bounds_s[:-1], bounds_s[1:]), ev_s):
+            main.wait_event(ev)
+            if b > a:
+                B.token_logprobs(d.hidden_s[a:b], self.w_vocab, d.ids_s[a:b], logprobs=lp_s[a:b], workspace=lm_ws,
+                                 device_status=self.status)
+                n_lm += 1
         main.wait_event(ev_suffix)
         B.suffix_attn(d.q_s, d.k_s, d.v_s, d.cu_suffix, d.prefix_lens, d.max_suffix_len, d.max_prefix_len, cache=cache,
                       out=o_s, workspace=attn_ws, device_status=self.status)
-        B.token_logprobs(d.hidden_s, self.w_vocab, d.ids_s, logprobs=lp_s, workspace=lm_ws, device_status=self.status)
         self._staging_free[turn] = t.cuda.Event()
         self._staging_free[turn].record(main)
         lp_p_host.copy_(lp_p, non_blocking=True)
         lp_s_host.copy_(lp_s, non_blocking=True)
-        self.kernels_last_host_pass = 2 + 2 * (sum(1 for a, b in zip(bounds[:-1], bounds[1:]) if b > a) + 1)
+        self.kernels_last_host_pass = 2 + 2 * n_lm
         return lp_p_host, lp_s_host
 
     def check_status(self) -> None:
