@@ -135,3 +135,31 @@ def test_a_sequence_longer_than_the_callers_bound_is_reported(cuda_device):
     rpx.prefix_attn(q, k, v, cu, 513, device_status=status)  # rounds up to 768: fine
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+
+
+def test_two_streams_with_their_own_workspaces_do_not_interfere(cuda_device):
+    """The library keeps no device state of its own: the attention kernel's work-item counter and the
+    LM head's partial records live in the caller's workspace, so calls on different streams with
+    different workspaces may overlap freely."""
+    dev = cuda_device
+    cfgs = [wk.Config("a", "bf16", 3, 4, 2, 128, 256, 3000, ("list", [700, 130, 257]), ("fixed", 0)),
+            wk.Config("b", "bf16", 2, 8, 1, 64, 128, 1000, ("list", [512, 300]), ("fixed", 0))]
+    wls = [wk.make_workload(c, seed=50 + i) for i, c in enumerate(cfgs)]
+    dev_in = [[to_device(x, dev) for x in (w.q, w.k, w.v, w.cu_full, w.hidden, w.w, w.ids)] for w in wls]
+
+    def run(i, stream):
+        q, k, v, cu, h, wv, ids = dev_in[i]
+        with torch.cuda.stream(stream):
+            o = rpx.prefix_attn(q, k, v, cu, int(wls[i].prompt_lens.max()))
+            lp = rpx.token_logprobs(h, wv, ids)
+        return o, lp
+
+    main = torch.cuda.current_stream()
+    ref = [run(i, main) for i in range(2)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for _ in range(3):
+        got = [run(i, streams[i]) for i in range(2)]
+        torch.cuda.synchronize()
+        for (ro, rl), (go, gl) in zip(ref, got):
+            assert torch.equal(ro, go) and torch.equal(rl, gl)
