@@ -127,7 +127,7 @@ class ScoringSession:
         mark(4)
         return lp_p, lp_s, o_p, o_s
 
-    def score_from_host(self, hb: Batch, lp_p_host, lp_s_host, lm_slices: int = 4):
+    def score_from_host(self, hb: Batch, lp_p_host, lp_s_host, lm_slices: int = 4, min_slice_rows: int = 2048):
         """Pinned host batch in, log-probs out into the pinned ``lp_*_host`` tensors.
 
         Host->device copies run on a copy stream in the order the kernels need them and each
@@ -175,9 +175,9 @@ class ScoringSession:
             rest = max(parts - (1 if first else 0), 1)
             return sorted(set([0] + [first + (n - first) * i // rest for i in range(rest + 1)]))
 
-        bounds_p = cut(n_p, lm_slices, True)
-        # response rows: slices of about the same size as the prompt-row slices, at most 8
-        bounds_s = cut(n_s, max(1, min(8, round(lm_slices * n_s / max(n_p, 1)), n_s // 4096)), False)
+        # no slice below min_slice_rows rows; response rows: slices of about the prompt-row slices' size, at most 8
+        bounds_p = cut(n_p, max(1, min(lm_slices, n_p // min_slice_rows)), True)
+        bounds_s = cut(n_s, max(1, min(8, round(lm_slices * n_s / max(n_p, 1)), n_s // (2 * min_slice_rows))), False)
         # Upload order = the order the kernels below consume their inputs.  The response rows of the LM
         # head run before the suffix attention (the two are independent), so that the large q/k/v of the
         # responses, needed last, also arrive last.
