@@ -178,17 +178,6 @@ class ScoringSession:
         # no slice below min_slice_rows rows; response rows: slices of about the prompt-row slices' size, at most 8
         bounds_p = cut(n_p, max(1, min(lm_slices, n_p // min_slice_rows)), True)
         bounds_s = cut(n_s, max(1, min(8, round(lm_slices * n_s / max(n_p, 1)), n_s // (2 * min_slice_rows))), False)
-        # Upload order = the order the kernels below consume their inputs.  The response rows of the LM
-        # head run before the suffix attention (the two are independent), so that the large q/k/v of the
-        # responses, needed last, also arrive last.
-        ev_ids = upload([(d.ids_p, hb.ids_p), (d.ids_s, hb.ids_s)])
-        ev_p = [upload([(d.hidden_p[a:b], hb.hidden_p[a:b])]) for a, b in zip(bounds_p[:-1], bounds_p[1:])]
-        ev_prefix = upload([(d.q_p, hb.q_p), (d.k_p, hb.k_p), (d.v_p, hb.v_p), (d.cu_prefix, hb.cu_prefix),
-                            (d.block_table, hb.block_table)])
-        ev_s = [upload([(d.hidden_s[a:b], hb.hidden_s[a:b])]) for a, b in zip(bounds_s[:-1], bounds_s[1:])]
-        ev_suffix = upload([(d.q_s, hb.q_s), (d.k_s, hb.k_s), (d.v_s, hb.v_s), (d.cu_suffix, hb.cu_suffix),
-                            (d.prefix_lens, hb.prefix_lens)])
-
         cache = (self.k_cache, self.v_cache, d.block_table)
         code = B._dtype_code(d.hidden_p)
         vocab, hdim = self.w_vocab.shape
@@ -201,26 +190,46 @@ class ScoringSession:
         attn_ws = self._workspace("attn", max(
             B.prefix_attn_workspace_bytes(d.q_p.shape[1], d.k_p.shape[1], d.q_p.shape[2], B._dtype_code(d.q_p), d.q_p.shape[0]),
             B.suffix_attn_workspace_bytes(d.q_s.shape[1], d.k_s.shape[1], d.q_s.shape[2], B._dtype_code(d.q_s), d.q_s.shape[0])))
+
+        def lm(hidden, ids, out, a, b):
+            def launch():
+                if b > a:
+                    B.token_logprobs(hidden[a:b], self.w_vocab, ids[a:b], logprobs=out[a:b], workspace=lm_ws,
+                                     device_status=self.status)
+                return 1 if b > a else 0
+            return launch
+
+        def attn_prefix():
+            B.prefix_attn(d.q_p, d.k_p, d.v_p, d.cu_prefix, d.max_prefix_len, cache=cache, out=o_p, workspace=attn_ws,
+                          device_status=self.status)
+            return 0
+
+        def attn_suffix():
+            B.suffix_attn(d.q_s, d.k_s, d.v_s, d.cu_suffix, d.prefix_lens, d.max_suffix_len, d.max_prefix_len,
+                          cache=cache, out=o_s, workspace=attn_ws, device_status=self.status)
+            return 0
+
+        # Stages = (what to upload, what to launch once it has landed), in the order the kernels run.  Each
+        # kernel is enqueued right behind its own upload, so the first one starts as soon as 15 MB have
+        # arrived; the copy stream runs the uploads back to back meanwhile.  The response rows of the LM head
+        # run before the suffix attention (the two are independent), so that the large q/k/v of the
+        # responses, needed last, also arrive last.
+        stages = []
+        for i, (a, b) in enumerate(zip(bounds_p[:-1], bounds_p[1:])):
+            pairs = [(d.hidden_p[a:b], hb.hidden_p[a:b])]
+            if i == 0:
+                pairs = [(d.ids_p, hb.ids_p), (d.ids_s, hb.ids_s)] + pairs
+            stages.append((pairs, lm(d.hidden_p, d.ids_p, lp_p, a, b)))
+        stages.append(([(d.q_p, hb.q_p), (d.k_p, hb.k_p), (d.v_p, hb.v_p), (d.cu_prefix, hb.cu_prefix),
+                        (d.block_table, hb.block_table)], attn_prefix))
+        for a, b in zip(bounds_s[:-1], bounds_s[1:]):
+            stages.append(([(d.hidden_s[a:b], hb.hidden_s[a:b])], lm(d.hidden_s, d.ids_s, lp_s, a, b)))
+        stages.append(([(d.q_s, hb.q_s), (d.k_s, hb.k_s), (d.v_s, hb.v_s), (d.cu_suffix, hb.cu_suffix),
+                        (d.prefix_lens, hb.prefix_lens)], attn_suffix))
         n_lm = 0
-        main.wait_event(ev_ids)
-        for (a, b), ev in zip(zip(bounds_p[:-1], bounds_p[1:]), ev_p):
-            main.wait_event(ev)
-            if b > a:
-                B.token_logprobs(d.hidden_p[a:b], self.w_vocab, d.ids_p[a:b], logprobs=lp_p[a:b], workspace=lm_ws,
-                                 device_status=self.status)
-                n_lm += 1
-        main.wait_event(ev_prefix)
-        B.prefix_attn(d.q_p, d.k_p, d.v_p, d.cu_prefix, d.max_prefix_len, cache=cache, out=o_p, workspace=attn_ws,
-                      device_status=self.status)
-        for (a, b), ev in zip(zip(bounds_s[:-1], bounds_s[1:]), ev_s):
-            main.wait_event(ev)
-            if b > a:
-                B.token_logprobs(d.hidden_s[a:b], self.w_vocab, d.ids_s[a:b], logprobs=lp_s[a:b], workspace=lm_ws,
-                                 device_status=self.status)
-                n_lm += 1
-        main.wait_event(ev_suffix)
-        B.suffix_attn(d.q_s, d.k_s, d.v_s, d.cu_suffix, d.prefix_lens, d.max_suffix_len, d.max_prefix_len, cache=cache,
-                      out=o_s, workspace=attn_ws, device_status=self.status)
+        for pairs, launch in stages:
+            main.wait_event(upload(pairs))
+            n_lm += launch()
         self._staging_free[turn] = t.cuda.Event()
         self._staging_free[turn].record(main)
         lp_p_host.copy_(lp_p, non_blocking=True)
