@@ -155,7 +155,7 @@ size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t tota
 
 size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype) {
     if (n_tokens <= 0 || hidden_dim <= 0 || vocab <= 0) return 0;
-    size_t bytes = align_up(static_cast<size_t>(logprob_num_chunks(vocab, logprob_tiles_per_chunk(n_tokens))) * n_tokens * sizeof(float4), kWsAlign);
+    size_t bytes = align_up(static_cast<size_t>(logprob_num_chunks(vocab, logprob_tiles_per_chunk(n_tokens, vocab))) * n_tokens * sizeof(float4), kWsAlign);
     if (dtype == RPX_F32) {
         bytes += align_up(static_cast<size_t>(n_tokens) * hidden_dim * 2, kWsAlign);
         bytes += align_up(static_cast<size_t>(vocab) * hidden_dim * 2, kWsAlign);
@@ -193,7 +193,7 @@ rpx_status_t run_token_logprobs(const void* hidden, int64_t hidden_row_stride, c
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     LogprobArgs a;
     a.partials = ws;
-    a.tiles_per_chunk = logprob_tiles_per_chunk(n_tokens);
+    a.tiles_per_chunk = logprob_tiles_per_chunk(n_tokens, vocab);
     ws += align_up(static_cast<size_t>(logprob_num_chunks(vocab, a.tiles_per_chunk)) * n_tokens * sizeof(float4), kWsAlign);
     a.hidden = hidden;
     a.hidden_row_stride = hidden_row_stride;

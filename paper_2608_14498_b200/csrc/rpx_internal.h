@@ -64,7 +64,7 @@ struct LogprobArgs {
     int32_t* device_status;
     cudaStream_t stream;
 };
-int32_t logprob_tiles_per_chunk(int64_t n_tokens);  // the default policy
+int32_t logprob_tiles_per_chunk(int64_t n_tokens, int32_t vocab);  // the default policy
 int32_t logprob_num_chunks(int32_t vocab, int32_t tiles_per_chunk);
 rpx_status_t launch_token_logprobs(const LogprobArgs& a);
 rpx_status_t launch_logprob_merge(const void* shard_stats, int32_t n_shards, const int32_t* target_ids, int64_t n_tokens,

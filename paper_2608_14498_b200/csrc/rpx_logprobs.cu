@@ -308,9 +308,26 @@ __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int3
 
 }  // namespace
 
-int32_t logprob_tiles_per_chunk(int64_t n_tokens) {
+int32_t logprob_tiles_per_chunk(int64_t n_tokens, int32_t vocab) {
     const int64_t row_tiles = (n_tokens + kBM - 1) / kBM;
-    if (row_tiles <= kSmallRowTiles) return kTilesPerChunkSmall;
+    if (row_tiles <= kSmallRowTiles) {
+        // Few row tiles mean few work items per CTA, so the last, partly filled round of items weighs in:
+        // take the chunk length (2..8 tiles) that needs the fewest tile-times on the part's 148 SMs, the
+        // longer one on a tie (fewer partial records).  This is pure arithmetic on the sizes, so that the
+        // workspace size can be computed without a device; on another SM count it is merely not tuned.
+        const int64_t vocab_tiles = (static_cast<int64_t>(vocab) + kBN - 1) / kBN;
+        int32_t best = kTilesPerChunkSmall;
+        int64_t best_cost = INT64_MAX;
+        for (int32_t tpc = 8; tpc >= 2; --tpc) {
+            const int64_t items = row_tiles * ((vocab_tiles + tpc - 1) / tpc);
+            const int64_t cost = ((items + 147) / 148) * tpc;
+            if (cost < best_cost) {
+                best_cost = cost;
+                best = tpc;
+            }
+        }
+        return best;
+    }
     return row_tiles >= kHugeRowTiles ? kTilesPerChunkHuge : kTilesPerChunkLarge;
 }
 

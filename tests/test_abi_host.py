@@ -62,8 +62,11 @@ def test_workspace_arithmetic(lib):
     assert B.token_logprobs_workspace_bytes(12800, 3584, 152064, B.RPX_BF16) == 38 * 12800 * 16
     assert B.token_logprobs_workspace_bytes(34816, 3584, 152064, B.RPX_BF16) == 75 * 34816 * 16
     f32 = B.token_logprobs_workspace_bytes(288, 256, 4096, B.RPX_F32)
-    # up to 64 row tiles the chunks are 4 vocabulary tiles long: 4096 columns = 16 tiles = 4 chunks
-    assert f32 == 4 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
+    # up to 64 row tiles the chunk length (2..8 tiles) is the one with the fewest rounds on 148 SMs:
+    # 3 row tiles x 16 vocabulary tiles -> 2-tile chunks, 8 of them
+    assert f32 == 8 * 288 * 16 + 288 * 256 * 2 + 4096 * 256 * 2
+    # 16 row tiles x 594 vocabulary tiles -> 5-tile chunks, 119 of them (65 tile-times against 64.2 ideal)
+    assert B.token_logprobs_workspace_bytes(2048, 3584, 152064, B.RPX_BF16) == 119 * 2048 * 16
     assert B.token_logprobs_workspace_bytes(0, 256, 4096, B.RPX_BF16) == 0
 
 
