@@ -584,6 +584,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         for (int i = 0; i < 32; ++i)
                             if (c * 32 + i >= n_vis) sc[c][i] = 0xff800000u;  // -inf
                 }
+                // keys no row of this warp may see (the upper right of a diagonal tile, the tail of the last
+                // prefix tile) need no exponentials: their 32-column chunks get P = 0 directly
+                const int32_t n_vis_warp = __reduce_max_sync(0xffffffffu, n_vis);
                 // eight independent chains: a row maximum is latency-bound, not throughput-bound
                 float mx[8];
 #pragma unroll
@@ -614,6 +617,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     for (int c = 0; c < kChunks; ++c) {
                         uint32_t packed[16];
                         uint32_t lo[4];
+                        if (c * 32 >= n_vis_warp) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) packed[i] = 0u;
+                            tmem_st16(my_s + c * 16, packed);
+                            if constexpr (kSplit) tmem_st16(my_s + 64 + c * 16, packed);
+                            continue;
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
                             const uint64_t x = f2_fma(
