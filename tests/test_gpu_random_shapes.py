@@ -34,7 +34,7 @@ def _draw(rng, case):
     return wk.Config(f"rand{case}", dtype, batch, group * hkv, hkv, d, hidden, vocab, ("list", plens), ("list", rlens))
 
 
-@pytest.mark.parametrize("case", range(12))
+@pytest.mark.parametrize("case", range(24))
 def test_random_batch_matches_the_oracle(cuda_device, case):
     dev = cuda_device
     rng = np.random.default_rng(1000 + case)
