@@ -20,13 +20,18 @@ rpx_status_t check_attn_desc(const rpx_attn_desc_t* d) {
     return RPX_OK;
 }
 
-// Layout: [work-item counter, kWsAlign bytes][RPX_F32 only: bf16 copies of q, k, v]
-size_t attn_workspace(const rpx_attn_desc_t* d, int64_t tokens) {
-    if (d == nullptr || tokens <= 0) return 0;
-    if (d->dtype != RPX_F32) return kWsAlign;
+// Layout: [work-item counter, kWsAlign bytes][RPX_F32 only: bf16 copies of q, k, v][suffix passes small enough
+// to be split over the cached prefix: split-KV partials]
+size_t attn_cast_workspace(const rpx_attn_desc_t* d, int64_t tokens) {
+    if (d->dtype != RPX_F32) return 0;
     const size_t qb = align_up(static_cast<size_t>(tokens) * d->num_q_heads * d->head_dim * 2, kWsAlign);
     const size_t kb = align_up(static_cast<size_t>(tokens) * d->num_kv_heads * d->head_dim * 2, kWsAlign);
-    return kWsAlign + qb + 2 * kb;
+    return qb + 2 * kb;
+}
+size_t attn_workspace(const rpx_attn_desc_t* d, int64_t tokens, bool is_suffix) {
+    if (d == nullptr || tokens <= 0) return 0;
+    return kWsAlign + attn_cast_workspace(d, tokens) +
+           (is_suffix ? attn_split_workspace(tokens, d->num_q_heads, d->head_dim) : 0);
 }
 
 rpx_status_t check_cache(const rpx_kv_cache_t* c, int32_t batch) {
@@ -59,7 +64,7 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     const int64_t kv_row = static_cast<int64_t>(desc->num_kv_heads) * desc->head_dim;
     if (q_tok_stride < q_row || k_tok_stride < kv_row || v_tok_stride < kv_row) return RPX_ERR_SHAPE;
     if (q_tok_stride % 8 || k_tok_stride % 8 || v_tok_stride % 8) return RPX_ERR_ALIGN;
-    const size_t need = attn_workspace(desc, total_tokens);
+    const size_t need = attn_workspace(desc, total_tokens, is_suffix);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return RPX_ERR_WORKSPACE;
     if (need > 0 && !aligned16(workspace)) return RPX_ERR_ALIGN;
     if (rpx_status_t rc = check_arch()) return rc;
@@ -101,6 +106,8 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.max_prefix_len = max_prefix_len;
     a.cache = cache;
     a.item_counter = static_cast<uint32_t*>(workspace);
+    if (is_suffix && attn_split_workspace(total_tokens, desc->num_q_heads, desc->head_dim) > 0)
+        a.split_ws = static_cast<uint8_t*>(workspace) + kWsAlign + attn_cast_workspace(desc, total_tokens);
     a.append_cache = is_suffix && append_cache;
     a.out = out;
     a.out_f32 = desc->dtype == RPX_F32;
@@ -136,7 +143,7 @@ rpx_status_t rpx_suffix_attn(const rpx_attn_desc_t* desc, const void* q, const v
 }
 
 size_t rpx_prefix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens) {
-    return attn_workspace(desc, total_tokens);
+    return attn_workspace(desc, total_tokens, false);
 }
 
 rpx_status_t rpx_chunk_attn(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
@@ -150,7 +157,7 @@ rpx_status_t rpx_chunk_attn(const rpx_attn_desc_t* desc, const void* q, const vo
 }
 
 size_t rpx_suffix_attn_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_suffix_tokens) {
-    return attn_workspace(desc, total_suffix_tokens);
+    return attn_workspace(desc, total_suffix_tokens, true);
 }
 
 size_t rpx_token_logprobs_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype) {

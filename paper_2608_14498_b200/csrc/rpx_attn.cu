@@ -33,6 +33,7 @@ namespace {
 
 constexpr int kTileQ = 128, kTileK = 128, kPage = 16;
 constexpr int kSlots = 4;  // K/V tiles in flight (two key steps); a fifth slot measured no faster
+constexpr int kMaxSplits = 4;  // ranges an item's cached prefix may be cut into
 constexpr int kItemRing = 4;  // work-item ids the producer may hand out ahead of the slowest warp
 constexpr int kChunks = kTileK / 32;  // 32-column TMEM loads per row and step
 constexpr int kWarpsPerTile = 4;
@@ -91,6 +92,13 @@ struct Params {
     int32_t n_pairs;              // query tile pairs per sequence the work list covers
     int32_t n_items;              // n_pairs * batch * num_q_heads
     uint32_t* next_item;          // device counter, zero before the launch: work items are handed out in order
+    // Split-KV (suffix passes with few, long items): the cached prefix of an item is cut into n_splits
+    // ranges taken by different CTAs; each writes an un-normalised partial, the last to arrive merges.
+    int32_t n_splits;             // 1 = off
+    float* part_o;                // [n_splits][tokens][H_q][D] fp32
+    float2* part_ml;              // [n_splits][tokens][H_q]: (row maximum in log2 units, row sum)
+    uint32_t* split_cnt;          // [tokens][H_q], zero before the launch: arrivals per 32-row group
+    int64_t total_tokens;
     float scale_log2;
     void* out;
     int32_t out_f32;
@@ -108,13 +116,16 @@ __device__ __forceinline__ uint32_t swz_off(int r, int cc) {
 // device counter, so the longest items start first and the short ones fill the tail.
 struct Item {
     int32_t pair, seq, head, kv_head, tok0, len_q, q0, len_p, n_prefix_tiles, n_tile0, n_kv;
+    int32_t pt0;      // first cached tile this item walks (n_prefix_tiles counts the tiles of its range)
+    int32_t x1;       // extra key steps of query tile 1 over tile 0: 1 when the item holds the self tiles, else 0
+    int32_t split, s_eff;  // which range of the cached prefix, out of how many (1 = the whole item)
     bool active, active1;
 };
 
 // The lengths come from device memory once per item (the producer's lane 0 reads them, a tile ahead of
 // everyone else, and passes them on through shared memory); the rest is arithmetic on the item number.
 __device__ __forceinline__ int4 fetch_item(const Params& p, int32_t idx) {
-    const int32_t seq = (idx % (p.batch * p.num_q_heads)) / p.num_q_heads;
+    const int32_t seq = ((idx / p.n_splits) % (p.batch * p.num_q_heads)) / p.num_q_heads;
     const int32_t tok0 = __ldg(p.cu_seqlens + seq);
     const int32_t len_q = __ldg(p.cu_seqlens + seq + 1) - tok0;
     const int32_t len_p = p.prefix_lens != nullptr ? __ldg(p.prefix_lens + seq) : 0;
@@ -128,7 +139,8 @@ __device__ __forceinline__ int4 read_item_rec(const int4* rec) {
 
 __device__ __forceinline__ Item decode_item(const Params& p, int4 rec) {
     Item it;
-    const int32_t idx = rec.x;
+    const int32_t idx = rec.x / p.n_splits;  // the item's (pair, sequence, head); its splits are numbered consecutively
+    it.split = rec.x % p.n_splits;
     const int32_t per_pair = p.batch * p.num_q_heads;
     it.pair = p.n_pairs - 1 - idx / per_pair;
     const int32_t rem = idx % per_pair;
@@ -141,12 +153,17 @@ __device__ __forceinline__ Item decode_item(const Params& p, int4 rec) {
     it.active = it.q0 < it.len_q;
     it.len_p = it.active ? rec.w : 0;
     it.active1 = it.q0 + kTileQ < it.len_q;
-    it.n_prefix_tiles = (it.len_p + kTileK - 1) / kTileK;
-    // key tiles seen by query tile t: n_tile0 + t.  (Scalars, not arrays: a small array indexed at
+    const int32_t n_pt = (it.len_p + kTileK - 1) / kTileK;  // cached tiles of the whole prefix
+    it.s_eff = max(1, min(p.n_splits, n_pt));                // a prefix shorter than n_splits tiles is cut in fewer
+    if (it.split >= it.s_eff) it.active = false;
+    it.pt0 = n_pt * min(it.split, it.s_eff) / it.s_eff;
+    it.n_prefix_tiles = n_pt * min(it.split + 1, it.s_eff) / it.s_eff - it.pt0;
+    it.x1 = it.split == it.s_eff - 1 ? 1 : 0;                // the last range also takes the self tiles
+    // key steps of query tile t: n_tile0 + t * x1.  (Scalars, not arrays: a small array indexed at
     // run time lives in local memory, and with nearly all L1 carved out as shared memory every such
     // load stalls the in-order warp for hundreds of cycles.)
-    it.n_tile0 = it.n_prefix_tiles + 2 * it.pair + 1;
-    it.n_kv = it.active1 ? it.n_tile0 + 1 : it.n_tile0;
+    it.n_tile0 = it.n_prefix_tiles + it.x1 * (2 * it.pair + 1);
+    it.n_kv = it.n_tile0 + (it.active1 ? it.x1 : 0);
     return it;
 }
 
@@ -249,10 +266,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (!it.active) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
-            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv, pt0 = it.pt0, x1 = it.x1;
             const bool active1 = it.active1;
             (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
-            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1; (void)pt0; (void)x1;
             // ---- Q of this item, once the previous item's last Q K^T has let go of the buffer
             if (n_active > 0 && !mbar_wait(&ctl->q_empty, (n_active - 1) & 1u, abort_flag)) {
                 ok = false;
@@ -280,10 +297,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 b = __ldg(p.block_table + static_cast<int64_t>(seq) * p.block_table_stride + page);
             return b;
         };
-        int32_t blk_next = n_prefix_tiles > 0 ? read_block_ids(0) : 0;
+        int32_t blk_next = n_prefix_tiles > 0 ? read_block_ids(pt0) : 0;
         for (int32_t j = 0; ok && j < n_kv; ++j) {
             const bool from_cache = j < n_prefix_tiles;
-            const int32_t jt = from_cache ? j : j - n_prefix_tiles;  // tile index inside its key source
+            const int32_t jt = from_cache ? pt0 + j : j - n_prefix_tiles;  // tile index inside its key source
             uint32_t slot_k = 0, slot_v = 0;
             int32_t blk = blk_next;  // this tile's pages (cached tiles only)
             if (from_cache) {
@@ -291,7 +308,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     ctl->data_error = 1;
                     blk = 0;
                 }
-                if (j + 1 < n_prefix_tiles) blk_next = read_block_ids(j + 1);
+                if (j + 1 < n_prefix_tiles) blk_next = read_block_ids(pt0 + j + 1);
             }
             for (int which = 0; which < 2; ++which, ++n_loaded) {  // 0 = K, 1 = V
                 const uint32_t slot = n_loaded % kSlots, phase = (n_loaded / kSlots) & 1u;
@@ -433,10 +450,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (!it.active) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
-            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv, pt0 = it.pt0, x1 = it.x1;
             const bool active1 = it.active1;
             (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
-            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1; (void)pt0; (void)x1;
             auto issue_qk = [&](int t, uint32_t k_slot) {
                 const uint64_t kd = k_desc0 + static_cast<uint64_t>(k_slot * (L::kKvBytes >> 4));
                 const uint64_t qd = q_desc0 + static_cast<uint64_t>(t * (L::kQBytes >> 4));
@@ -448,7 +465,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
                 const uint64_t vd = v_desc0 + static_cast<uint64_t>(v_slot * (L::kKvBytes >> 4));
                 umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128, vd, idesc_pv, accumulate ? 1u : 0u);
-                if (n_tile0 + t <= 2)  // + P_lo V, P_lo in columns 64..127 of S_t
+                if (it.s_eff == 1 && n_tile0 + t <= 2)  // + P_lo V, P_lo in columns 64..127 of S_t
                     umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128 + 64, vd, idesc_pv, 1u);
             };
 
@@ -467,7 +484,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const uint32_t v_slot = v_idx % kSlots, kn_slot = kn_idx % kSlots;
                 bool have_v = false, have_kn = false;
                 for (int t = 0; t < 2 && ok; ++t) {
-                    if ((t == 1 && !active1) || j >= n_tile0 + t) continue;
+                    if ((t == 1 && !active1) || j >= n_tile0 + t * x1) continue;
                     if (!mbar_wait(&ctl->p_ready[t], ((t ? cnt1 : cnt0) + j) & 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -489,7 +506,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     }
                     tc_fence_after_sync();
                     issue_pv(t, v_slot, j != 0);
-                    if (j + 1 < n_tile0 + t) {
+                    if (j + 1 < n_tile0 + t * x1) {
                         if (!have_kn) {
                             if (!mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag)) {
                                 ok = false;
@@ -512,7 +529,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             kv_base += 2u * static_cast<uint32_t>(n_kv);
             cnt0 += static_cast<uint32_t>(n_tile0);
             if (active1) {
-                cnt1 += static_cast<uint32_t>(n_tile0) + 1u;
+                cnt1 += static_cast<uint32_t>(n_tile0 + x1);
                 ++items1;
             }
             ++n_active;
@@ -542,15 +559,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (!it.active || (t == 1 && !it.active1)) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
-            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv;
+            const int32_t n_tile0 = it.n_tile0, n_kv = it.n_kv, pt0 = it.pt0, x1 = it.x1;
             const bool active1 = it.active1;
             (void)pair; (void)seq; (void)head; (void)kv_head; (void)tok0; (void)len_q; (void)q0; (void)len_p;
-            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1;
+            (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1; (void)pt0; (void)x1;
             const uint32_t quarter = warp & 3;
             const int32_t row = quarter * 32 + lane;
             const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
             const uint32_t lane_addr = (quarter * 32u) << 16;
-            const int32_t my_tiles = n_tile0 + t;
+            const int32_t my_tiles = n_tile0 + t * x1;
             const uint32_t my_s = tmem_base + t * 128 + lane_addr;        // this thread's lane of S_t / P_t
             const uint32_t my_o = tmem_base + 256 + t * 128 + lane_addr;  // and of O_t
             float run_max = -CUDART_INF_F, run_sum = 0.f;
@@ -572,7 +589,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // ---- how many leading keys of this tile the row may see
                 int32_t n_vis;
                 if (j < n_prefix_tiles) {
-                    n_vis = min(kTileK, len_p - j * kTileK);
+                    n_vis = min(kTileK, len_p - (pt0 + j) * kTileK);
                 } else {
                     const int32_t jt = j - n_prefix_tiles;
                     n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
@@ -676,7 +693,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(&ctl->p_ready[t]);
               }
             };
-            if (my_tiles <= 2)
+            if (it.s_eff == 1 && my_tiles <= 2)
                 run_steps(std::true_type{});
             else
                 run_steps(std::false_type{});
@@ -687,7 +704,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (ok) {
                 tc_fence_after_sync();
                 const bool row_valid = q_local < len_q;
-                const float inv = 1.f / run_sum;
+                float inv = 1.f / run_sum;
                 const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
                 // two chunks of 32 columns in flight: the next chunk's TMEM load runs under this chunk's stores
                 uint32_t ra[32], rb[32];
@@ -728,6 +745,85 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         }
                     }
                 };
+                if (it.s_eff > 1) {
+                    // ---- one range of a split item: the un-normalised row and its (maximum, sum) go to the
+                    // workspace; whichever of the s_eff CTAs arrives last for these 32 rows merges them
+                    const int64_t rh = static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head;
+                    const int64_t per_split = p.total_tokens * p.num_q_heads;
+                    float* po = p.part_o + (static_cast<int64_t>(it.split) * per_split + rh) * D;
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(my_o + c * 32, ra);
+                        tmem_ld_wait();
+                        if (c == D / 32 - 1) {  // O_t is out of TMEM
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&ctl->o_free[t]);
+                        }
+                        if (row_valid) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                st_global_v8(po + c * 32 + 8 * i, ra[8 * i], ra[8 * i + 1], ra[8 * i + 2], ra[8 * i + 3],
+                                             ra[8 * i + 4], ra[8 * i + 5], ra[8 * i + 6], ra[8 * i + 7]);
+                        }
+                    }
+                    const bool warp_valid = q0 + t * kTileQ + static_cast<int32_t>(quarter) * 32 < len_q;  // lane 0's row
+                    if (row_valid) p.part_ml[static_cast<int64_t>(it.split) * per_split + rh] = make_float2(run_max, run_sum);
+                    uint32_t arrived = 0;
+                    if (warp_valid) {
+                        __threadfence();
+                        __syncwarp();
+                        if (lane == 0)
+                            arrived = atomicAdd(p.split_cnt + (static_cast<int64_t>(tok0 + q0 + t * kTileQ) + quarter * 32) *
+                                                                  p.num_q_heads + head, 1u);
+                        arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    }
+                    if (warp_valid && arrived == static_cast<uint32_t>(it.s_eff - 1)) {
+                        __threadfence();
+                        float f[kMaxSplits];
+                        float top = -CUDART_INF_F, total = 0.f;
+                        if (row_valid) {
+#pragma unroll
+                            for (int sp = 0; sp < kMaxSplits; ++sp)
+                                if (sp < it.s_eff)
+                                    top = fmaxf(top, __ldcg(p.part_ml + static_cast<int64_t>(sp) * per_split + rh).x);
+                            total = 0.f;
+#pragma unroll
+                            for (int sp = 0; sp < kMaxSplits; ++sp) {
+                                if (sp < it.s_eff) {
+                                    const float2 ml = __ldcg(p.part_ml + static_cast<int64_t>(sp) * per_split + rh);
+                                    f[sp] = fast_exp2(ml.x - top);
+                                    total = fmaf(f[sp], ml.y, total);
+                                } else {
+                                    f[sp] = 0.f;
+                                }
+                            }
+                            inv = 1.f / total;
+#pragma unroll 1
+                            for (int c = 0; c < D / 32; ++c) {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) ra[i] = 0u;
+#pragma unroll
+                                for (int sp = 0; sp < kMaxSplits; ++sp) {
+                                    if (sp < it.s_eff) {
+                                        const float4* src = reinterpret_cast<const float4*>(
+                                            p.part_o + (static_cast<int64_t>(sp) * per_split + rh) * D + c * 32);
+#pragma unroll
+                                        for (int i = 0; i < 8; ++i) {
+                                            const float4 v = __ldcg(src + i);
+                                            ra[4 * i] = __float_as_uint(fmaf(f[sp], v.x, __uint_as_float(ra[4 * i])));
+                                            ra[4 * i + 1] = __float_as_uint(fmaf(f[sp], v.y, __uint_as_float(ra[4 * i + 1])));
+                                            ra[4 * i + 2] = __float_as_uint(fmaf(f[sp], v.z, __uint_as_float(ra[4 * i + 2])));
+                                            ra[4 * i + 3] = __float_as_uint(fmaf(f[sp], v.w, __uint_as_float(ra[4 * i + 3])));
+                                        }
+                                    }
+                                }
+                                store_chunk(ra, c);
+                            }
+                            if (p.lse != nullptr) p.lse[rh] = (top + log2f(total)) * kLn2;
+                        }
+                    }
+                } else {
                 tmem_ld32(my_o, ra);
 #pragma unroll
                 for (int c = 0; c < D / 32; c += 2) {
@@ -748,6 +844,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 }
                 if (row_valid && p.lse != nullptr)
                     p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
+                }
             }
         }
     }
@@ -813,15 +910,47 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.out_f32 = a.out_f32 ? 1 : 0;
     p.lse = a.lse;
     p.status = a.device_status;
-    const int64_t n_items = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
-    if (n_items <= 0) return RPX_OK;
+    const int64_t n_base = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
+    if (n_base <= 0) return RPX_OK;
+    int sms_all = sm_count();
+    if (sms_all <= 0) return RPX_ERR_CUDA;
+    if (const int budget = sm_budget(); budget > 0 && budget < sms_all) sms_all = budget;
+    // ---- split-KV: a suffix pass with few, long items leaves most SMs idle in its last round of items.
+    // Cutting the cached prefix of every item into S ranges gives S times as many, shorter items; taken when
+    // the estimated number of key steps on the busiest SM drops by more than 15 %.
+    p.n_splits = 1;
+    p.part_o = nullptr;
+    p.part_ml = nullptr;
+    p.split_cnt = nullptr;
+    p.total_tokens = a.total_tokens;
+    if (a.prefix_lens != nullptr && p.write_cache == 0 && a.split_ws != nullptr &&
+        attn_split_workspace(a.total_tokens, a.num_q_heads, D) > 0) {
+        const int64_t prefix_steps = (a.max_prefix_len + kTileK - 1) / kTileK;
+        const int64_t self_steps = 2 * p.n_pairs + 1;
+        // rounds of items x (key steps + about four steps' worth of fixed cost per item); with three ranges on C2's
+        // suffix pass (224 items of 35 steps) the merge and the fixed costs ate the gain: 0.219 against 0.156 ms
+        auto cost = [&](int64_t S) { return ((n_base * S + sms_all - 1) / sms_all) * (prefix_steps / S + 4) + self_steps; };
+        int best = 1;
+        for (int S = 2; S <= kMaxSplits; ++S)
+            if (prefix_steps / S >= 4 && cost(S) < cost(best)) best = S;
+        if (best > 1 && cost(best) * 100 < cost(1) * 85) {
+            p.n_splits = best;
+            const size_t rows = static_cast<size_t>(a.total_tokens) * a.num_q_heads;
+            uint8_t* ws = static_cast<uint8_t*>(a.split_ws);
+            p.split_cnt = reinterpret_cast<uint32_t*>(ws);
+            ws += (rows * sizeof(uint32_t) + 255) / 256 * 256;
+            p.part_ml = reinterpret_cast<float2*>(ws);
+            ws += (kMaxSplits * rows * sizeof(float2) + 255) / 256 * 256;
+            p.part_o = reinterpret_cast<float*>(ws);
+            if (cudaMemsetAsync(p.split_cnt, 0, rows * sizeof(uint32_t), a.stream) != cudaSuccess) return RPX_ERR_CUDA;
+        }
+    }
+    const int64_t n_items = n_base * p.n_splits;
     if (n_items > INT32_MAX - 65536) return RPX_ERR_SHAPE;  // the counter runs past n_items by one draw per CTA
     if (a.item_counter == nullptr) return RPX_ERR_WORKSPACE;
     p.n_items = static_cast<int32_t>(n_items);
     p.next_item = a.item_counter;
-    int sms = sm_count();
-    if (sms <= 0) return RPX_ERR_CUDA;
-    if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;  // leave the rest to a co-runner
+    const int sms = sms_all;  // SM count, or the caller's SM budget: the rest is left to a co-runner
     const int64_t grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM
     if (cudaMemsetAsync(a.item_counter, 0, sizeof(uint32_t), a.stream) != cudaSuccess) return RPX_ERR_CUDA;
     if (cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -832,6 +961,15 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
 }
 
 }  // namespace
+
+size_t attn_split_workspace(int64_t tokens, int32_t num_q_heads, int32_t head_dim) {
+    // worth splitting only while the items (256 rows each) do not fill the SMs a few times over anyway
+    const int64_t rows = tokens * num_q_heads;
+    if (tokens <= 0 || rows > 3 * 148 * 2 * kTileQ) return 0;
+    const size_t r = static_cast<size_t>(rows);
+    return (r * sizeof(uint32_t) + 255) / 256 * 256 + (kMaxSplits * r * sizeof(float2) + 255) / 256 * 256 +
+           (kMaxSplits * r * head_dim * sizeof(float) + 255) / 256 * 256;
+}
 
 rpx_status_t launch_attention(const AttnArgs& a) {
     if (a.total_tokens == 0 || a.batch == 0 || a.max_q_len == 0) return RPX_OK;

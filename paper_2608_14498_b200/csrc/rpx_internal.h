@@ -39,6 +39,7 @@ struct AttnArgs {
     const rpx_kv_cache_t* cache;       // prefix pass: written (nullable); suffix pass: read
     bool append_cache = false;         // chunked prefill: read the earlier chunks AND append this one
     uint32_t* item_counter = nullptr;  // 4 bytes of workspace: the kernel's work-item counter (zeroed by the launcher)
+    void* split_ws = nullptr;          // suffix pass only: room for split-KV partials (attn_split_workspace bytes), or NULL
     void* out;
     bool out_f32;
     float* lse;
@@ -46,6 +47,9 @@ struct AttnArgs {
     cudaStream_t stream;
 };
 rpx_status_t launch_attention(const AttnArgs& a);
+// Split-KV workspace of a suffix pass over `tokens` query tokens: arrival counters, (max, sum) pairs and fp32
+// partial rows for up to 4 ranges; 0 when the pass is too large to ever be split.
+size_t attn_split_workspace(int64_t tokens, int32_t num_q_heads, int32_t head_dim);
 
 struct LogprobArgs {
     const void* hidden;   // bf16 [n][hidden_row_stride]

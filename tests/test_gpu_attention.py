@@ -142,6 +142,28 @@ def test_prefix_without_cache_and_explicit_scale(cuda_device):
     assert err <= TOL
 
 
+def test_suffix_pass_split_over_the_cached_prefix(cuda_device):
+    """Few, long work items: the launcher cuts every item's cached prefix into ranges taken by different
+    CTAs and the last to arrive merges the partial rows.  Mixed prefix lengths: 32 tiles (4 ranges), one
+    tile (not split), 20 tiles with a ragged last one; ragged response lengths leave warps without rows."""
+    cfg = wk.Config("t", "bf16", 3, 4, 2, 128, 64, 64, ("list", [4000, 100, 2500]), ("list", [200, 300, 64]))
+    wl = wk.make_workload(cfg, seed=17, lm=False)
+    out, lse, kc, vc, (p1, s1) = run_split(wl, cuda_device)
+    rows = oracle.all_rows(wl.cu_full, cfg.num_q_heads)
+    suffix_only = rows[rows[:, 1] >= wl.prompt_lens[rows[:, 0]]]
+    check_rows(wl, out, lse, suffix_only)
+    check_rows(wl, out, lse, sample_prefix_rows(wl, rows))
+    # the merge order of the ranges depends on which CTA arrives last, the merged bits do not
+    _, _, _, _, (p2, s2) = run_split(wl, cuda_device)
+    assert torch.equal(s1, s2)
+
+
+def sample_prefix_rows(wl, rows, n=400):
+    pre = rows[rows[:, 1] < wl.prompt_lens[rows[:, 0]]]
+    pick = np.random.default_rng(5).choice(pre.shape[0], size=min(n, pre.shape[0]), replace=False)
+    return pre[np.sort(pick)]
+
+
 def test_sm_budget_changes_no_bit_of_the_attention_outputs(cuda_device):
     cfg = wk.Config("t", "bf16", 3, 4, 2, 128, 64, 64, ("list", [600, 333, 48]), ("list", [100, 20, 260]))
     wl = wk.make_workload(cfg, seed=15, lm=False)
