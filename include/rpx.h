@@ -119,7 +119,7 @@ RPX_API rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q,
  * 0..r; the result equals rows prefix_lens[s].. of one-pass attention over the whole sequence.
  *   q, k, v: response tokens only, packed by cu_seqlens_suffix; prefix_lens device int32 [batch]
  *   cache: required, read-only here (response K/V are NOT appended; they have no later reader)
- *   workspace: rpx_suffix_attn_workspace_bytes includes, for passes of up to 227 328 (token, head) rows,
+ *   workspace: rpx_suffix_attn_workspace_bytes includes, for passes of up to 113 664 (token, head) rows,
  *   room for split-KV partials: when the batch is a few long items, the cached prefix of each is cut
  *   into ranges worked on by different SMs and merged by the last to finish (same result up to fp32
  *   rounding of the merge, identical from run to run).
