@@ -158,6 +158,15 @@ def test_suffix_pass_split_over_the_cached_prefix(cuda_device):
     assert torch.equal(s1, s2)
 
 
+def test_suffix_pass_split_in_two_with_head_dim_64(cuda_device):
+    """Nine cached tiles at most: two ranges; a 3-tile prefix is cut 1 + 2, a sequence without prefix not at all."""
+    cfg = wk.Config("t", "bf16", 3, 8, 1, 64, 64, 64, ("list", [1100, 300, 0]), ("list", [130, 256, 40]))
+    wl = wk.make_workload(cfg, seed=18, lm=False)
+    out, lse, kc, vc, _ = run_split(wl, cuda_device)
+    check_rows(wl, out, lse, oracle.all_rows(wl.cu_full, cfg.num_q_heads))
+    check_cache(wl, kc, vc)
+
+
 def sample_prefix_rows(wl, rows, n=400):
     pre = rows[rows[:, 1] < wl.prompt_lens[rows[:, 0]]]
     pick = np.random.default_rng(5).choice(pre.shape[0], size=min(n, pre.shape[0]), replace=False)
