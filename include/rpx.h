@@ -14,9 +14,13 @@
  *     (rpx_attn_desc_t, rpx_kv_cache_t) are read on the HOST during the call.
  *   - The caller owns every buffer (inputs, outputs, cache pool, block table, workspace, status
  *     word) and must keep it alive until `cuda_stream` has executed the enqueued work.  The
- *     library allocates no device memory, keeps no state between calls and never synchronises:
- *     a call only enqueues kernels on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
- *     legacy default stream) of the current device.
+ *     library allocates no device memory, keeps no state between calls (but see
+ *     rpx_set_sm_budget) and never synchronises: a call only enqueues kernels, and small
+ *     asynchronous memsets of its workspace, on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream) of the current device.
+ *   - A workspace belongs to one call at a time: the kernels keep their work-item counters and
+ *     partial results there, so two calls that may overlap on the GPU (different streams) need
+ *     different workspaces.  Calls on one stream may share one.
  *   - Packed layouts: a [tokens][heads][head_dim] tensor has head_dim contiguous, heads
  *     contiguous (stride head_dim) and a caller-given token stride in ELEMENTS.  Sequence s owns
  *     tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (int32, device, batch+1 entries, cu_seqlens[0]=0).
