@@ -100,6 +100,7 @@ struct Params {
     uint32_t* split_cnt;          // [tokens][H_q], zero before the launch: arrivals per 32-row group
     int64_t total_tokens;
     float scale_log2;
+    float inv_scale_log2;
     void* out;
     int32_t out_f32;
     float* lse;
@@ -604,21 +605,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // keys no row of this warp may see (the upper right of a diagonal tile, the tail of the last
                 // prefix tile) need no exponentials: their 32-column chunks get P = 0 directly
                 const int32_t n_vis_warp = __reduce_max_sync(0xffffffffu, n_vis);
-                // eight independent chains: a row maximum is latency-bound, not throughput-bound
+                // eight independent chains of three-input maxima (the maximum runs on the half-rate ALU pipe,
+                // so halving its instruction count is worth more than it looks)
                 float mx[8];
+                auto score = [&](int e) { return __uint_as_float(sc[e >> 5][e & 31]); };
 #pragma unroll
-                for (int u = 0; u < 8; ++u) mx[u] = -CUDART_INF_F;
+                for (int u = 0; u < 8; ++u) mx[u] = fmaxf(score(u), score(8 + u));
 #pragma unroll
-                for (int c = 0; c < kChunks; ++c)
+                for (int e = 16; e < kTileK; e += 16)
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8)
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(sc[c][i + u]));
-                float cmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                                   fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                    for (int u = 0; u < 8; ++u) mx[u] = fmax3(mx[u], score(e + u), score(e + 8 + u));
+                float cmax = fmax3(fmax3(mx[0], mx[1], mx[2]), fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
                 cmax *= p.scale_log2;  // scale > 0, so max commutes with the scaling
+                // The running maximum is kept integer-valued (rounded up): any upper bound serves the softmax, and
+                // an integer maximum can be folded exactly into the rounding constant of the polynomial exp2 below.
                 const bool grow = cmax > run_max + kRescaleThreshold;
-                const float new_max = grow ? cmax : run_max;
+                const float new_max = grow ? ceilf(cmax) : run_max;
                 const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
                 const bool rescale = j > 0 && __any_sync(0xffffffffu, grow);
                 run_sum *= alpha;
@@ -626,6 +628,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // ---- P = 2^(x - max) as packed bf16 pairs over the first 64 columns of S_t
                 const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
                 const uint64_t neg_max2 = f2_pack(-run_max, -run_max);
+                const uint64_t magic_max2 = f2_pack(12582912.f - run_max, 12582912.f - run_max);
+                const float min_score = (run_max - 125.f) * p.inv_scale_log2;
                 uint64_t part2[4] = {0ull, 0ull, 0ull, 0ull};  // four packed accumulators = eight chains
                 // kSplit also writes the second bf16 term of each probability (what the first term's
                 // rounding dropped) to columns 64..127, four words at a time to keep it in registers.
@@ -643,15 +647,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                         }
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const uint64_t x = f2_fma(
-                                f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])), scale2, neg_max2);
                             float e0, e1;
-                            float x0, x1;
-                            f2_unpack(x, x0, x1);
                             if (((i / 2) % 4) < kPolyPairsOf4) {  // compile-time per unrolled pair
-                                e0 = poly_exp2(x0);  // scalar form: its constants are immediates, the packed
-                                e1 = poly_exp2(x1);  // form would pin seven register pairs in this loop
+                                // exp2 on the FMA pipe, with the scaling folded in: s * scale + (1.5 * 2^23 - max)
+                                // rounds x = s * scale - max to the integer n in its low mantissa bits (the
+                                // maximum is an integer, so the constant is exact); f = x - n by a second FMA;
+                                // 2^f by a cubic; 2^n goes into the exponent field.  Scores are clamped so that
+                                // x >= -125 (masked ones are -inf): the result is then at most 2^-125.
+                                const uint64_t sp = f2_pack(fmaxf(__uint_as_float(sc[c][i]), min_score),
+                                                            fmaxf(__uint_as_float(sc[c][i + 1]), min_score));
+                                const uint64_t shifted = f2_fma(sp, scale2, magic_max2);
+                                const uint64_t f = f2_fma(sp, scale2, f2_sub(magic_max2, shifted));
+                                uint64_t pf = f2_fma(f2_pack(0.05500858f, 0.05500858f), f, f2_pack(0.24221037f, 0.24221037f));
+                                pf = f2_fma(pf, f, f2_pack(0.6932829f, 0.6932829f));
+                                pf = f2_fma(pf, f, f2_pack(1.0f, 1.0f));
+                                float p0, p1, s0, s1;
+                                f2_unpack(pf, p0, p1);
+                                f2_unpack(shifted, s0, s1);
+                                e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(s0) << 23));
+                                e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(s1) << 23));
                             } else {
+                                const uint64_t x = f2_fma(
+                                    f2_pack(__uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1])), scale2, neg_max2);
+                                float x0, x1;
+                                f2_unpack(x, x0, x1);
                                 e0 = fast_exp2(x0);
                                 e1 = fast_exp2(x1);
                             }
@@ -906,6 +925,7 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.n_pairs = (a.max_q_len + 2 * kTileQ - 1) / (2 * kTileQ);
     const float scale = a.softmax_scale > 0.f ? a.softmax_scale : 1.0f / sqrtf(static_cast<float>(D));
     p.scale_log2 = scale * kLog2e;
+    p.inv_scale_log2 = 1.0f / p.scale_log2;
     p.out = a.out;
     p.out_f32 = a.out_f32 ? 1 : 0;
     p.lse = a.lse;
