@@ -125,11 +125,22 @@ struct Item {
 
 // The lengths come from device memory once per item (the producer's lane 0 reads them, a tile ahead of
 // everyone else, and passes them on through shared memory); the rest is arithmetic on the item number.
-__device__ __forceinline__ int4 fetch_item(const Params& p, int32_t idx) {
+// Offsets that do not describe a range inside the packed tensors (a negative length, an end beyond total_tokens, a
+// negative cached length, more pages than a row of the block table holds) are reported and the item is handed on
+// empty, so nothing is read or written through them.
+__device__ __forceinline__ int4 fetch_item(const Params& p, int32_t idx, uint32_t* data_error) {
     const int32_t seq = ((idx / p.n_splits) % (p.batch * p.num_q_heads)) / p.num_q_heads;
     const int32_t tok0 = __ldg(p.cu_seqlens + seq);
-    const int32_t len_q = __ldg(p.cu_seqlens + seq + 1) - tok0;
-    const int32_t len_p = p.prefix_lens != nullptr ? __ldg(p.prefix_lens + seq) : 0;
+    int32_t len_q = __ldg(p.cu_seqlens + seq + 1) - tok0;
+    int32_t len_p = p.prefix_lens != nullptr ? __ldg(p.prefix_lens + seq) : 0;
+    // pages the block table must hold for this sequence: its cached prefix, plus its own tokens where they are stored
+    const int64_t table_tokens = static_cast<int64_t>(len_p) + (p.write_cache != 0 ? len_q : 0);
+    if (tok0 < 0 || len_q < 0 || static_cast<int64_t>(tok0) + len_q > p.total_tokens || len_p < 0 ||
+        (p.block_table != nullptr && (table_tokens + kPage - 1) / kPage > p.block_table_stride)) {
+        *data_error = 1;
+        len_q = 0;
+        len_p = 0;
+    }
     return make_int4(idx, tok0, len_q, len_p);
 }
 
@@ -251,7 +262,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             int4 rec = make_int4(-1, 0, 0, 0);
             if (lane == 0) {
                 const int32_t idx = static_cast<int32_t>(atomicAdd(p.next_item, 1u));
-                if (idx < p.n_items) rec = fetch_item(p, idx);
+                if (idx < p.n_items) rec = fetch_item(p, idx, &ctl->data_error);
                 ctl->item_rec[ring] = rec;
                 mbar_arrive(&ctl->item_full[ring]);
             }
@@ -483,7 +494,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             for (int32_t j = 0; ok && j < n_kv; ++j) {
                 const uint32_t v_idx = kv_base + 2 * j + 1, kn_idx = kv_base + 2 * j + 2;
                 const uint32_t v_slot = v_idx % kSlots, kn_slot = kn_idx % kSlots;
-                bool have_v = false, have_kn = false;
+                // V_j and K_{j+1} were asked for a step ago: make sure of them BEFORE waiting for the probabilities, so
+                // that the tensor core starts the moment the softmax warps arrive
+                const bool have_kn = j + 1 < n_kv;
+                if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag) ||
+                    (have_kn && !mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag))) {
+                    ok = false;
+                    break;
+                }
                 for (int t = 0; t < 2 && ok; ++t) {
                     if ((t == 1 && !active1) || j >= n_tile0 + t * x1) continue;
                     if (!mbar_wait(&ctl->p_ready[t], ((t ? cnt1 : cnt0) + j) & 1u, abort_flag)) {
@@ -498,24 +516,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                             break;
                         }
                     }
-                    if (!have_v) {
-                        if (!mbar_wait(&ctl->kv_full[v_slot], (v_idx / kSlots) & 1u, abort_flag)) {
-                            ok = false;
-                            break;
-                        }
-                        have_v = true;
-                    }
                     tc_fence_after_sync();
                     issue_pv(t, v_slot, j != 0);
                     if (j + 1 < n_tile0 + t * x1) {
-                        if (!have_kn) {
-                            if (!mbar_wait(&ctl->kv_full[kn_slot], (kn_idx / kSlots) & 1u, abort_flag)) {
-                                ok = false;
-                                break;
-                            }
-                            tc_fence_after_sync();
-                            have_kn = true;
-                        }
                         issue_qk(t, kn_slot);  // in order behind PV_t(j): P_t is read before S_t is rewritten
                     } else {
                         umma_commit(&ctl->o_done[t]);

@@ -163,3 +163,36 @@ def test_two_streams_with_their_own_workspaces_do_not_interfere(cuda_device):
         torch.cuda.synchronize()
         for (ro, rl), (go, gl) in zip(ref, got):
             assert torch.equal(ro, go) and torch.equal(rl, gl)
+
+
+def test_sequence_offsets_that_leave_the_packed_tensors_are_reported_not_followed(cuda_device):
+    """cu_seqlens live on the device, so the host cannot check them: an end beyond total_tokens, or offsets that run
+    backwards, must raise RPX_ERR_DEVICE_DATA and must not make the kernel store outside the output tensor."""
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 3, 4, 2, 128, 64, 64, ("list", [150, 70, 40]), ("list", [0, 0, 0]))
+    wl = wk.make_workload(cfg, seed=44, lm=False)
+    qp, kp, vp = (to_device(wl.prefix_pack(t), dev) for t in (wl.q, wl.k, wl.v))
+    total = qp.shape[0]
+    ref_out = rpx.prefix_attn(qp, kp, vp, to_device(wl.cu_prefix, dev), 150)
+    torch.cuda.synchronize()
+    # the output tensor sits in the middle of a guard region filled with a recognisable value
+    guard = torch.full((3 * total, 4, 128), 7.0, dtype=torch.bfloat16, device=dev)
+    out = guard[total:2 * total]
+    for bad in ([0, 150, 220, total + 300],      # the last sequence claims 300 tokens more than exist
+                [0, 150, 120, total],            # offsets run backwards: sequence 1 has a negative length
+                [0, 150, 220, -5]):              # a negative end
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        guard.fill_(7.0)
+        cu = torch.tensor(bad, dtype=torch.int32, device=dev)
+        rpx.prefix_attn(qp, kp, vp, cu, 512, out=out, device_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == -8, bad
+        assert bool((guard[:total] == 7.0).all()) and bool((guard[2 * total:] == 7.0).all()), bad
+        # sequence 0 is well-formed in every case and is still computed (in the second case the third sequence,
+        # tokens 120..259, overlaps its last rows)
+        assert torch.equal(out[:120], ref_out[:120]), bad
+    # the context is intact and a well-formed call is clean afterwards
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    again = rpx.prefix_attn(qp, kp, vp, to_device(wl.cu_prefix, dev), 150, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(again, ref_out)
