@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the prefix+suffix scoring hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3]
+    python bench.py --profile-case lm|prefix|suffix [--reps 3]      (small launches for profiler captures)
 
 One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
 boundary-KV write), prefix log-probs, suffix attention over the cached KV, suffix log-probs.
@@ -15,6 +16,10 @@ Metric: scored tokens/s (every token of every sequence gets a log-prob) and TFLO
             / its CUDA-event duration, against the measured dense-bf16 peak of this machine.
 `cpu_baseline`  the fp64 oracle, as it stands, on a bounded sample of the same workload.
 `--impl reference` times that oracle alone (rank 0 only).
+
+The headline workload is C3 (the largest single-GPU config: 32 packed sequences of the 32B shape, the
+paper's main setup); with one GPU the line also carries a `configs` record with C2, C4 and C5 measured
+the same way in the same invocation (fewer steps each, own clock samples).
 
 N > 1 (torchrun): every rank scores its own batch of the same shape (sequences are independent,
 W_vocab replicated, no data-path collective) => weak scaling; time = max over ranks.
@@ -39,9 +44,8 @@ if ROOT not in sys.path:
 from paper_2608_14498_b200 import workloads as wk  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the LM-head partial kernel on the
-# benchmark's prompt-row launch (32768 x 152064 x 3584), from a one-pass ncu capture of this very
-# command; summary in profiles/lm_head_partial_kernel__slice_8192x32768x3584.md.  Other configs: None.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the LM-head partial kernel on a config's
+# prompt rows, from one-pass ncu captures of this very command on that config.  Configs without a capture: None.
 LM_HEAD_TRAFFIC_BYTES = {"C2": 13.291e9 + 43.8e6}
 
 
@@ -195,26 +199,21 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, rank, local_rank, world):
-    import torch
-    import torch.distributed as dist
-
+def measure_config(torch, dist, config, steps, warmup, rank, local_rank, world, cpu_tokens=0):
+    """Times one config on this rank's GPU: device-resident steps with events around every call, then the
+    end-to-end path from pinned host memory (synchronised per step, and with the caller one step behind).
+    Rank 0 gets the result record (the others None).  Clocks are sampled while the timed regions run."""
     import paper_2608_14498_b200 as rpx
+    from paper_2608_14498_b200.dist import job_throughput
     from paper_2608_14498_b200.pipeline import KERNELS_PER_SCORE, Batch, ScoringSession
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
-    rpx.load_library()
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
 
     def barrier():
         if world > 1:
             dist.barrier()
 
-    cfg = wk.CONFIGS[args.config]
+    cfg = wk.CONFIGS[config]
     wl = wk.make_workload(cfg, seed=rank)
     flops = flop_counts(wl)
     hb = host_batch(wl, torch)
@@ -225,7 +224,7 @@ def run_ours(args, rank, local_rank, world):
     lp_p_host = torch.empty(wl.n_prefix, dtype=torch.float32).pin_memory()
     lp_s_host = torch.empty(wl.n_suffix, dtype=torch.float32).pin_memory()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         sess.score(db)
     torch.cuda.synchronize()
     sess.check_status()
@@ -240,19 +239,19 @@ def run_ours(args, rank, local_rank, world):
 
     # ---------------- device-resident timing: events around every call of every step
     names = ["prefix_attn", "lm_prefix", "suffix_attn", "lm_suffix"]
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
     barrier()
     torch.cuda.synchronize()
     if sampler:
         sampler.mark()
-    for s in range(args.steps):
+    for s in range(steps):
         sess.score(db, events=ev[s])
     torch.cuda.synchronize()
     if sampler:
         sampler.mark()
     barrier()
     total_ms = ev[0][0].elapsed_time(ev[-1][4])
-    per_kernel_ms = {n: sum(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps)) / args.steps
+    per_kernel_ms = {n: sum(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(steps)) / steps
                      for i, n in enumerate(names)}
     sess.check_status()
 
@@ -263,7 +262,7 @@ def run_ours(args, rank, local_rank, world):
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         sess.score_from_host(hb, lp_p_host, lp_s_host)
         torch.cuda.current_stream().synchronize()  # the caller consumes the log-probs every step
     e1.record()
@@ -278,7 +277,7 @@ def run_ours(args, rank, local_rank, world):
     barrier()
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record()
-    for i in range(args.steps):
+    for i in range(steps):
         if i >= 2:
             done[i & 1].synchronize()  # step i-2's results have landed and been consumed: its buffers are free
         sess.score_from_host(hb, *host_sets[i & 1])
@@ -289,71 +288,158 @@ def run_ours(args, rank, local_rank, world):
     sess.check_status()
     clocks = sampler.stop() if sampler else None
 
-    from paper_2608_14498_b200.dist import job_throughput
-
     job_tokens, total_ms = job_throughput(wl.n_tokens, total_ms, dev)
     job_suffix, e2e_ms = job_throughput(wl.n_suffix, e2e_ms, dev)
     _, e2e_pipelined_ms = job_throughput(wl.n_tokens, e2e_pipelined_ms, dev)
+    if rank != 0:
+        return None
 
+    peaks = load_peaks()
+    ms_per_step = total_ms / steps
+    total_flops = sum(flops.values())
+    step_s = ms_per_step * 1e-3
+    # a step is seconds of back-to-back tensor work at the power cap: the sustained peak applies
+    peak_tf = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    burst_tf = float(peaks["bf16_tflops"])
+    lm_ms = per_kernel_ms["lm_prefix"]
+    lm_tf = flops["lm_prefix"] / (lm_ms * 1e-3) / 1e12
+    kernels = {}
+    for n in names:
+        tf = flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12
+        kernels[n] = {"ms": round(per_kernel_ms[n], 4), "tflops": round(tf, 1),
+                      "frac_of_sustained_peak": round(tf / peak_tf, 4), "frac_of_burst_peak": round(tf / burst_tf, 4),
+                      "frac_of_datasheet_dense_bf16": round(tf / 2250.0, 4)}
+    gb = lambda n: f"{n / 1e9:.2f} GB"
+    rec = {
+        "value": job_tokens / step_s, "ms_per_step": ms_per_step,
+        "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "prompt_tokens": wl.n_prefix,
+                   "response_tokens": wl.n_suffix, "scored_tokens_per_gpu": wl.n_tokens, "q_heads": cfg.num_q_heads,
+                   "kv_heads": cfg.num_kv_heads, "head_dim": cfg.head_dim, "hidden": cfg.hidden, "vocab": cfg.vocab,
+                   "kv_block": 16, "parallelism": f"dp{world} (independent sequences per rank, no collective)",
+                   "l2": f"no flush: per-step inputs (W_vocab {gb(wl.w.nbytes)}, hidden {gb(wl.hidden.nbytes)}, "
+                         f"Q/K/V {gb(wl.q.nbytes + wl.k.nbytes + wl.v.nbytes)}) exceed the 126 MB L2",
+                   "stands_in_for": cfg.stands_in_for},
+        "tflops": total_flops * world / step_s / 1e12,
+        "frac_of_sustained_peak": total_flops / step_s / 1e12 / peak_tf,
+        "frac_of_burst_peak": total_flops / step_s / 1e12 / burst_tf,
+        "response_tokens_per_s": job_suffix / step_s,
+        "kernels": kernels,
+        "roofline": {"kernel": "lm_head_partial_kernel (prompt rows; event pair spans it and its 0.1 % combine kernel)",
+                     "bound": "tensor", "achieved": lm_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": lm_tf / peak_tf,
+                     "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
+                     "frac_of_burst_peak": lm_tf / burst_tf,
+                     "traffic": LM_HEAD_TRAFFIC_BYTES.get(config),
+                     "algorithmic_bytes": (wl.n_prefix * cfg.hidden + cfg.vocab * cfg.hidden) * 2 + 8 * wl.n_prefix},
+        "e2e": {"value": job_tokens / (e2e_ms / steps * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": hb.nbytes(), "d2h_bytes_per_step": (wl.n_prefix + wl.n_suffix) * 4,
+                "ms_per_step": e2e_ms / steps,
+                "note": "the stream is synchronised after every step; with the caller one step behind "
+                        "(double-buffered results) a step takes pipelined_ms_per_step.  Only the log-probs come "
+                        "back to the host: the attention outputs O_p / O_s stay on the device by design (they "
+                        "feed the next layer there), so they are not part of d2h_bytes_per_step",
+                "pipelined_ms_per_step": e2e_pipelined_ms / steps},
+        "gpu_launches": KERNELS_PER_SCORE * steps,
+        "gpu_launches_e2e": sess.kernels_last_host_pass * steps,
+        "clocks": clocks,
+        "steps": steps,
+    }
+    if world == 1 and cpu_tokens > 0:
+        import oracle
+
+        oracle.build()
+        t = oracle_sample(wl, cpu_tokens, 0)
+        rec["cpu_baseline"] = {
+            "value": cpu_tokens / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{cpu_tokens} tokens drawn uniformly from the batch ({cfg.num_q_heads} attention rows + 1 log-prob row each), {t:.1f} s"}
+    return rec
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2608_14498_b200 as rpx
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
+    rpx.load_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    head = measure_config(torch, dist, args.config, args.steps, args.warmup, rank, local_rank, world,
+                          cpu_tokens=0 if args.no_cpu_baseline else args.cpu_tokens)
+    others = {}
+    if world == 1 and not args.no_sub_configs:
+        # the other bf16 configs, measured the same way (fewer steps; their own clock samples)
+        for name in ("C2", "C4", "C5"):
+            if name == args.config:
+                continue
+            torch.cuda.empty_cache()
+            sub = measure_config(torch, dist, name, max(5, args.steps // 3), args.warmup, rank, local_rank, world)
+            others[name] = {k: sub[k] for k in ("value", "ms_per_step", "steps", "tflops", "frac_of_sustained_peak",
+                                                "frac_of_burst_peak", "kernels", "e2e", "clocks")}
+            others[name]["workload"] = sub["config"]["workload"]
     if rank == 0:
-        peaks = load_peaks()
-        ms_per_step = total_ms / args.steps
-        value = job_tokens / (ms_per_step * 1e-3)
-        total_flops = sum(flops.values())
-        step_s = ms_per_step * 1e-3
-        # a step is seconds of back-to-back tensor work at the power cap: the sustained peak applies
-        peak_tf = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-        lm_ms = per_kernel_ms["lm_prefix"]
-        lm_tf = flops["lm_prefix"] / (lm_ms * 1e-3) / 1e12
-        kernels = {}
-        for n in names:
-            tf = flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12
-            kernels[n] = {"ms": round(per_kernel_ms[n], 4), "tflops": round(tf, 1),
-                          "frac_of_sustained_peak": round(tf / peak_tf, 4),
-                          "frac_of_burst_peak": round(tf / float(peaks["bf16_tflops"]), 4)}
         line = {
-            "metric": "scored_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": "scored_tokens_per_s", "value": head["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "prompt_tokens": wl.n_prefix,
-                       "response_tokens": wl.n_suffix, "scored_tokens_per_gpu": wl.n_tokens, "q_heads": cfg.num_q_heads,
-                       "kv_heads": cfg.num_kv_heads, "head_dim": cfg.head_dim, "hidden": cfg.hidden, "vocab": cfg.vocab,
-                       "kv_block": 16, "parallelism": f"dp{world} (independent sequences per rank, no collective)",
-                       "l2": "no flush: per-step inputs (W_vocab 1.09 GB, hidden 0.25 GB, Q/K/V 0.32 GB) exceed the 126 MB L2",
-                       "stands_in_for": cfg.stands_in_for},
-            "tflops": total_flops * world / step_s / 1e12,
-            "frac_of_bf16_peak": total_flops / step_s / 1e12 / peak_tf,
-            "response_tokens_per_s": job_suffix / step_s,
-            "kernels": kernels,
-            "roofline": {"kernel": "lm_head_partial_kernel (prompt rows; event pair spans it and its 0.1 % combine kernel)",
-                         "bound": "tensor", "achieved": lm_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": lm_tf / peak_tf,
-                         "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
-                         "frac_of_burst_peak": lm_tf / float(peaks["bf16_tflops"]),
-                         "traffic": LM_HEAD_TRAFFIC_BYTES.get(args.config),
-                         "algorithmic_bytes": (wl.n_prefix * cfg.hidden + cfg.vocab * cfg.hidden) * 2 + 8 * wl.n_prefix},
-            "e2e": {"value": job_tokens / (e2e_ms / args.steps * 1e-3), "unit": "tokens/s",
-                    "h2d_bytes_per_step": hb.nbytes(), "d2h_bytes_per_step": (wl.n_prefix + wl.n_suffix) * 4,
-                    "ms_per_step": e2e_ms / args.steps,
-                    "note": "the stream is synchronised after every step; with the caller one step behind "
-                            "(double-buffered results) a step takes pipelined_ms_per_step",
-                    "pipelined_ms_per_step": e2e_pipelined_ms / args.steps},
-            "gpu_launches": KERNELS_PER_SCORE * args.steps,
-            "gpu_launches_e2e": sess.kernels_last_host_pass * args.steps,
-            "clocks": clocks,
         }
-        if world == 1 and not args.no_cpu_baseline:
-            import oracle
-
-            oracle.build()
-            n = args.cpu_tokens
-            t = oracle_sample(wl, n, 0)
-            line["cpu_baseline"] = {
-                "value": n / t, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-                "sample": f"{n} tokens drawn uniformly from the batch ({cfg.num_q_heads} attention rows + 1 log-prob row each), {t:.1f} s"}
+        line.update({k: v for k, v in head.items() if k not in ("value", "ms_per_step", "steps")})
+        if others:
+            line["configs"] = others
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_profile_case(args):
+    """Small, self-terminating launches of one kernel for profiler captures.  Each case keeps a few hundred MB on
+    the device (more than the 126 MB L2, so DRAM counters mean something) and launches the kernel `reps` times
+    after one warm-up launch.
+      lm      8192 rows x 32768 vocabulary columns, hidden 3584  (7B-shaped slice of the LM head)
+      prefix  4 sequences x 4096 prompt tokens, 28 query / 4 KV heads, head_dim 128, with cache write
+      suffix  the same 4 prompts cached, 256 response tokens each"""
+    import torch
+
+    import paper_2608_14498_b200 as rpx
+
+    dev = torch.device("cuda:0")
+
+    def dv(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+        return torch.from_numpy(a).to(dev)
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    case = args.profile_case
+    if case == "lm":
+        cfg = wk.Config("profile-lm", "bf16", 1, 28, 4, 128, 3584, 32768, ("fixed", 8192), ("fixed", 0))
+        wl = wk.make_workload(cfg, seed=0, attn=False)
+        h, w, ids = dv(wl.hidden), dv(wl.w), dv(wl.ids)
+        for _ in range(1 + args.reps):
+            rpx.token_logprobs(h, w, ids, device_status=status)
+    else:
+        cfg = wk.Config("profile-attn", "bf16", 4, 28, 4, 128, 3584, 1024, ("fixed", 4096), ("fixed", 256))
+        wl = wk.make_workload(cfg, seed=0, lm=False)
+        kc = torch.zeros((wl.num_blocks, 4, 16, 128), dtype=torch.bfloat16, device=dev)
+        cache = (kc, torch.zeros_like(kc), dv(wl.block_table))
+        qp, kp, vp = (dv(wl.prefix_pack(t)) for t in (wl.q, wl.k, wl.v))
+        qs, ks, vs = (dv(wl.suffix_pack(t)) for t in (wl.q, wl.k, wl.v))
+        cu_p, cu_s, pl = dv(wl.cu_prefix), dv(wl.cu_suffix), dv(wl.prompt_lens)
+        rpx.prefix_attn(qp, kp, vp, cu_p, 4096, cache=cache, device_status=status)
+        for _ in range(args.reps + (1 if case == "suffix" else 0)):
+            if case == "prefix":
+                rpx.prefix_attn(qp, kp, vp, cu_p, 4096, cache=cache, device_status=status)
+            else:
+                rpx.suffix_attn(qs, ks, vs, cu_s, pl, 256, 4096, cache=cache, device_status=status)
+    torch.cuda.synchronize()
+    code = int(status.item())
+    if code != 0:
+        raise SystemExit(f"device status {code}: {rpx.status_string(code)}")
+    print(f"profile case {case}: ok")
 
 
 def run_group(args):
@@ -420,10 +506,13 @@ def run_group(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))
+    ap.add_argument("--config", default="C3", choices=sorted(wk.CONFIGS), help="headline workload (C3 = the largest single-GPU config)")
+    ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
+    ap.add_argument("--profile-case", choices=["lm", "prefix", "suffix"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -432,7 +521,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.group > 0:
+    if args.profile_case:
+        if rank == 0:
+            run_profile_case(args)
+    elif args.group > 0:
         if rank == 0:
             run_group(args)
     elif args.impl == "reference":

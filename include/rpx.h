@@ -31,11 +31,13 @@
  *   - Host-checkable problems (NULL pointer, head counts, head_dim, block size, alignment,
  *     strides, workspace size, device architecture) return a negative status BEFORE any launch.
  *     Problems only visible on the device (a kernel-side wait that ran out, an out-of-range
- *     target id or block id) are written to *device_status (nullable, device int32, zeroed by the
+ *     target id or block id, sequence offsets that run backwards or past the end of the packed
+ *     tensors, a sequence with more pages than a row of the block table) are written to *device_status (nullable, device int32, zeroed by the
  *     caller): the first error code wins; the caller reads it after its own synchronisation.
  *     Every kernel-side wait is bounded: on expiry the kernel records RPX_ERR_TIMEOUT, drains and
  *     returns; outputs of that call are then undefined.
- *   - Alignment: every tensor pointer 16-byte aligned; token/row strides multiples of 8 elements.
+ *   - Alignment: every tensor pointer 16-byte aligned; token/row strides multiples of 8 elements;
+ *     every workspace pointer 256-byte aligned (RPX_ERR_ALIGN otherwise, before any launch).
  *   - Zero-length sequences, batch == 0 and n_tokens == 0 are legal no-ops.
  */
 #ifndef RPX_H_
@@ -96,8 +98,9 @@ typedef struct {
 } rpx_kv_cache_t;
 
 /*
- * Prefix attention + boundary-KV write (Section 3.1, Phase 1: "prefill the prompt ... produces
- * ... boundary KV state").  For every sequence s, query head h and prompt position i:
+ * Prefix attention + boundary-KV write (Section 3.1, Phase 1: the prompt is prefilled before any
+ * response exists, which leaves behind the KV state at the prompt/response boundary).  For every
+ * sequence s, query head h and prompt position i:
  *     out[i,h,:] = sum_{j<=i} softmax_j(scale * q[i,h,:].k[j,g,:]) * v[j,g,:],   g = h / group
  * and, when `cache` is non-NULL, K and V of every prompt token are stored (as bf16) at the
  * token's slot of the paged cache; slots no token maps to are not touched.
@@ -116,9 +119,9 @@ RPX_API rpx_status_t rpx_prefix_attn(const rpx_attn_desc_t* desc, const void* q,
                              void* cuda_stream);
 
 /*
- * Suffix attention over the retained boundary (Section 3.1, Phase 2: "suffixes consume the
- * responses and their preserved boundaries"; Section 2.3: they "continue from the retained prefix
- * boundary rather than recomputing the prompt").  Response position r of sequence s (global
+ * Suffix attention over the retained boundary (Section 3.1, Phase 2: the suffix pass takes the
+ * responses together with the boundary state kept from Phase 1; Section 2.3: the prompt is not
+ * computed a second time).  Response position r of sequence s (global
  * position prefix_lens[s] + r) attends to all prefix_lens[s] cached keys and to response keys
  * 0..r; the result equals rows prefix_lens[s].. of one-pass attention over the whole sequence.
  *   q, k, v: response tokens only, packed by cu_seqlens_suffix; prefix_lens device int32 [batch]
@@ -159,8 +162,8 @@ RPX_API rpx_status_t rpx_chunk_attn(const rpx_attn_desc_t* desc, const void* q, 
                             size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
 /*
- * Fused LM-head log-probabilities (Section 3.1: Phase 1 yields "prefix log-probabilities",
- * Phase 2 the suffix ones; Table 4 "Prefix logprobs").  For every row n:
+ * Fused LM-head log-probabilities (Section 3.1: Phase 1 yields the log-probabilities of the prefix
+ * positions, Phase 2 those of the suffix; Table 4, row on prefix log-probabilities).  For every row n:
  *     z_v = hidden[n,:] . w_vocab[v,:]          (never stored)
  *     logprobs[n] = z_{target_ids[n]} - ln sum_v exp(z_v)
  *   hidden [n_tokens][hidden_dim] with row stride in elements; w_vocab [vocab][hidden_dim]
@@ -221,7 +224,9 @@ RPX_API rpx_status_t rpx_token_logprobs_merge(const float* shard_stats, int32_t 
  * The per-(vocab chunk, row) partial records that rpx_token_logprobs keeps in the caller's
  * workspace live here in a fixed array of RPX_STATIC_SCRATCH_BYTES inside the library image;
  * every GPU that loads the library holds that array until the process exits.  Inputs and outputs
- * are still the caller's.  bf16 inputs only; same result as rpx_token_logprobs.
+ * are still the caller's.  bf16 inputs only; the result equals that of rpx_token_logprobs up to the order in
+ * which fp32 partial sums are merged (this entry point always cuts the vocabulary into 16-tile chunks, the
+ * workspace variant into 2 to 16 tiles depending on the row count).
  *   - Limit: ceil(ceil(vocab / 256) / 16) * n_tokens * 16 bytes must not exceed
  *     RPX_STATIC_SCRATCH_BYTES (vocab 152064 => at most 13797 rows per call); larger problems
  *     return RPX_ERR_WORKSPACE before any launch — split the rows over several calls.

@@ -170,7 +170,26 @@ def _workspace(nbytes: int, device, workspace):
         if workspace.numel() * workspace.element_size() < nbytes:
             raise ValueError(f"workspace too small: need {nbytes} bytes")
         return workspace
-    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device=device)
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def _in_call_context(fn):
+    """Runs a wrapper with its first tensor's device current (the library launches on the current device) and,
+    when ``stream=`` is given, with that stream current, so that outputs and temporary workspaces the wrapper
+    allocates belong to the stream the kernels run on."""
+    import functools
+
+    @functools.wraps(fn)
+    def call(*args, **kwargs):
+        torch = _torch()
+        first = args[0] if args else next(iter(kwargs.values()))
+        stream = kwargs.get("stream")
+        with torch.cuda.device(first.device):
+            if stream is None:
+                return fn(*args, **kwargs)
+            with torch.cuda.stream(stream):
+                return fn(*args, **kwargs)
+    return call
 
 
 def _desc(q, k, softmax_scale: float) -> AttnDesc:
@@ -222,6 +241,7 @@ def get_sm_budget() -> int:
 
 
 # ------------------------------------------------------------------ the three calls
+@_in_call_context
 def prefix_attn(q, k, v, cu_seqlens, max_seqlen: int, cache: Optional[Tuple] = None, softmax_scale: float = 0.0,
                 out=None, lse=None, return_lse: bool = False, workspace=None, device_status=None, stream=None):
     """rpx_prefix_attn: causal GQA attention over packed prompts, writing the paged KV cache.
@@ -248,6 +268,7 @@ def prefix_attn(q, k, v, cu_seqlens, max_seqlen: int, cache: Optional[Tuple] = N
     return (out, lse) if return_lse else out
 
 
+@_in_call_context
 def suffix_attn(q, k, v, cu_seqlens_suffix, prefix_lens, max_suffix_len: int, max_prefix_len: int, cache: Tuple,
                 softmax_scale: float = 0.0, out=None, lse=None, return_lse: bool = False, workspace=None,
                 device_status=None, stream=None):
@@ -272,6 +293,7 @@ def suffix_attn(q, k, v, cu_seqlens_suffix, prefix_lens, max_suffix_len: int, ma
     return (out, lse) if return_lse else out
 
 
+@_in_call_context
 def chunk_attn(q, k, v, cu_seqlens_chunk, cached_lens, max_chunk_len: int, max_cached_len: int, cache: Tuple,
                 softmax_scale: float = 0.0, out=None, lse=None, return_lse: bool = False, workspace=None,
                 device_status=None, stream=None):
@@ -297,6 +319,7 @@ def chunk_attn(q, k, v, cu_seqlens_chunk, cached_lens, max_chunk_len: int, max_c
     return (out, lse) if return_lse else out
 
 
+@_in_call_context
 def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_lse: bool = False, workspace=None,
                    device_status=None, stream=None, entropy=None):
     """rpx_token_logprobs: log p(target) per row from hidden [N, H] and W [V, H]; logits never stored.
@@ -331,6 +354,7 @@ def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_
     return (logprobs, lse) if return_lse else logprobs
 
 
+@_in_call_context
 def token_logprobs_static(hidden, w_vocab, target_ids, logprobs, lse=None, device_status=None, stream=None):
     """rpx_token_logprobs_static: the same log-probs, for callers that cannot allocate device memory.
 
@@ -356,6 +380,7 @@ def token_logprobs_static(hidden, w_vocab, target_ids, logprobs, lse=None, devic
     return logprobs
 
 
+@_in_call_context
 def token_logprobs_shard(hidden, w_shard, target_ids, vocab_begin: int, shard_stats=None, workspace=None,
                          device_status=None, stream=None):
     """rpx_token_logprobs_shard: this rank's share of a vocabulary-parallel LM head.
@@ -382,6 +407,7 @@ def token_logprobs_shard(hidden, w_shard, target_ids, vocab_begin: int, shard_st
     return shard_stats
 
 
+@_in_call_context
 def token_logprobs_merge(all_stats, target_ids, vocab_total: int, logprobs=None, return_lse: bool = False, entropy=None,
                          device_status=None, stream=None):
     """rpx_token_logprobs_merge: final log-probs from the gathered shard records float32 [R, N, 4]."""

@@ -26,29 +26,72 @@ from __future__ import annotations
 import argparse
 import json
 import statistics
+import subprocess
+import threading
+import time
 
 import numpy as np
 
 
-def main() -> None:
+class _Clocks:
+    """SM clock and throttle reasons sampled with nvidia-smi (read-only) while a measurement runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int = 0, period_s: float = 0.1):
+        self.index, self.period_s, self.rows, self._stop = index, period_s, [], threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                self.rows.append([x.strip() for x in out.strip().split(",")])
+            except (OSError, subprocess.SubprocessError):
+                return
+            self._stop.wait(self.period_s)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        mhz = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "", 1).isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in self.rows if len(r) >= 6 for n, v in zip(names, r[2:6]) if v.lower() == "active"})
+        sm_max = next((float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "", 1).isdigit()), None)
+        return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": sm_max, "reasons": reasons,
+                "samples": len(mhz)}
+
+
+def run(config: str = "C2", ratios=(0.5, 1.0, 2.0), reps: int = 5, decode_gb: float = 4.0, sm_budgets=(0,), workload=None,
+        emit=print):
+    """Runs the measurement and returns its records (one per SM budget and decode length); `emit` gets each as a
+    JSON line.  `workload` overrides the named config (used by the tests with a tiny one).  Also returns, under
+    "check", what the scoring pass produced during the last co-run, so a caller can compare it with the oracle."""
     import torch
 
     from . import binding as B
     from . import workloads as wk
     from .pipeline import ScoringSession
 
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))
-    ap.add_argument("--ratios", type=float, nargs="+", default=[0.5, 1.0, 2.0], help="target T_D / T_P")
-    ap.add_argument("--reps", type=int, default=5)
-    ap.add_argument("--decode-gb", type=float, default=4.0, help="weight bytes one decode step streams")
-    ap.add_argument("--sm-budgets", type=int, nargs="+", default=[0], help="LM-head CTA caps to sweep (0 = none)")
-    args = ap.parse_args()
+    class _Args:
+        pass
+
+    args = _Args()
+    args.ratios, args.reps, args.decode_gb, args.sm_budgets = list(ratios), reps, decode_gb, list(sm_budgets)
     dev = torch.device("cuda", 0)
     B.load_library()
 
-    cfg = wk.CONFIGS[args.config]
-    wl = wk.make_workload(cfg, seed=0)
+    wl = workload if workload is not None else wk.make_workload(wk.CONFIGS[config], seed=0)
+    cfg = wl.cfg
+    records = []
 
     def t(a):
         x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
@@ -113,8 +156,9 @@ def main() -> None:
         sess.check_status()
         for ratio in args.ratios:
             steps = max(1, round(ratio * t_p / t_step))
-            _, t_d = median(False, steps)
-            t_p_co, t_d_co = median(True, steps)
+            with _Clocks() as clk:
+                _, t_d = median(False, steps)
+                t_p_co, t_d_co = median(True, steps)
             delta_d = t_d_co - t_d
             makespan = max(t_d_co, t_p_co)
             line = {
@@ -127,10 +171,27 @@ def main() -> None:
                 # S_measured is the prefix work's own slowdown under co-run
                 "S_eq1_ms": t_d + t_p - max(t_d + delta_d, t_p),
                 "serial_ms": t_d + t_p, "overlapped_ms": makespan, "speedup": (t_d + t_p) / makespan,
+                "clocks": clk.summary(),
             }
-            print(json.dumps(line), flush=True)
+            records.append(line)
+            emit(json.dumps(line))
     B.set_sm_budget(0)
     sess.check_status()
+    torch.cuda.synchronize()
+    return {"records": records, "check": {"out": out, "logprobs": lp, "prefix_rows": pre}}
+
+
+def main() -> None:
+    from . import workloads as wk
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="C2", choices=sorted(wk.CONFIGS))
+    ap.add_argument("--ratios", type=float, nargs="+", default=[0.5, 1.0, 2.0], help="target T_D / T_P")
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--decode-gb", type=float, default=4.0, help="weight bytes one decode step streams")
+    ap.add_argument("--sm-budgets", type=int, nargs="+", default=[0], help="LM-head CTA caps to sweep (0 = none)")
+    args = ap.parse_args()
+    run(args.config, args.ratios, args.reps, args.decode_gb, args.sm_budgets, emit=lambda s: print(s, flush=True))
 
 
 if __name__ == "__main__":

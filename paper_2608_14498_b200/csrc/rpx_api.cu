@@ -11,6 +11,8 @@ using namespace rpx;
 constexpr size_t kWsAlign = 256;
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// Workspaces are carved in 256-byte pieces that the kernels access with vector loads and stores of up to 32 bytes.
+bool aligned_ws(const void* p) { return (reinterpret_cast<uintptr_t>(p) & (kWsAlign - 1)) == 0; }
 
 rpx_status_t check_attn_desc(const rpx_attn_desc_t* d) {
     if (d == nullptr) return RPX_ERR_NULL;
@@ -66,7 +68,7 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     if (q_tok_stride % 8 || k_tok_stride % 8 || v_tok_stride % 8) return RPX_ERR_ALIGN;
     const size_t need = attn_workspace(desc, total_tokens, is_suffix);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return RPX_ERR_WORKSPACE;
-    if (need > 0 && !aligned16(workspace)) return RPX_ERR_ALIGN;
+    if (need > 0 && !aligned_ws(workspace)) return RPX_ERR_ALIGN;
     if (rpx_status_t rc = check_arch()) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
@@ -193,7 +195,7 @@ rpx_status_t run_token_logprobs(const void* hidden, int64_t hidden_row_stride, c
     if (!aligned16(hidden) || !aligned16(w_vocab) || !aligned16(shard_stats)) return RPX_ERR_ALIGN;
     const size_t need = rpx_token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype);
     if (workspace == nullptr || workspace_bytes < need) return RPX_ERR_WORKSPACE;
-    if (!aligned16(workspace)) return RPX_ERR_ALIGN;
+    if (!aligned_ws(workspace)) return RPX_ERR_ALIGN;
     if (rpx_status_t rc = check_arch()) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 

@@ -53,12 +53,20 @@ def job_throughput(local_units: float, local_ms: float, device=None) -> Tuple[fl
 
 
 def vocab_shard_bounds(vocab: int, world_size: int, rank: int, multiple: int = 256):
-    """[begin, end) of the vocabulary rows rank `rank` holds: equal shares rounded to `multiple`
-    columns (one LM-head tile), the last rank taking the remainder (possibly empty-free: >= 1)."""
-    per = -(-vocab // world_size)
-    per = -(-per // multiple) * multiple
-    begin = min(vocab, rank * per)
-    end = vocab if rank == world_size - 1 else min(vocab, begin + per)
+    """[begin, end) of the vocabulary rows rank `rank` holds.  The vocabulary is cut into tiles of `multiple`
+    rows (one LM-head tile; the last may be partial) and the tiles are dealt out as evenly as they go, in order.
+
+    Every rank must hold at least one row: an empty shard has no work for rpx_token_logprobs_shard
+    (it rejects vocab_local == 0) while the other ranks would wait for it in the all-gather.  A vocabulary
+    with fewer tiles than ranks therefore raises ValueError; pass a smaller `multiple`."""
+    if world_size <= 0 or not 0 <= rank < world_size:
+        raise ValueError("rank must lie in [0, world_size)")
+    tiles = -(-vocab // multiple)
+    if tiles < world_size:
+        raise ValueError(f"a vocabulary of {vocab} rows has {tiles} tiles of {multiple} rows: not enough to give "
+                         f"each of {world_size} ranks a non-empty shard")
+    begin = (tiles * rank // world_size) * multiple
+    end = vocab if rank == world_size - 1 else (tiles * (rank + 1) // world_size) * multiple
     return begin, end
 
 

