@@ -57,6 +57,11 @@ def _load():
         lib.rpx_oracle_cache_image.restype = ctypes.c_int
         lib.rpx_oracle_cache_image.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, i32, i32, i32, vp, i32,
                                                i32, i64, vp, vp]
+        lib.rpx_oracle_logprob_backward.restype = ctypes.c_int
+        lib.rpx_oracle_logprob_backward.argtypes = [vp, i64, vp, ctypes.c_int, vp, vp, i64, i32, i32, vp, vp]
+        lib.rpx_oracle_attn_backward.restype = ctypes.c_int
+        lib.rpx_oracle_attn_backward.argtypes = [vp, vp, vp, ctypes.c_int, i64, i64, i64, vp, i32, i32, i32, i32, dbl,
+                                                 vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -187,3 +192,51 @@ def cache_image(k, v, cu_seqlens, block_table, num_blocks: int, block_size: int 
     if rc != 0:
         raise ValueError(f"rpx_oracle_cache_image failed with {rc}")
     return kc, vc
+
+
+def logprob_backward(hidden, w, target_ids, upstream, want_dw: bool = False):
+    """Gradient of sum_n upstream[n] * logprob[n] with respect to hidden (and to w when asked), from the definition
+    dL/dz = upstream * (onehot(target) - softmax(z)) in fp64.  hidden [N, H], w [V, H], target_ids int32 [N],
+    upstream float64 [N].  Returns dhidden float64 [N, H] (and dw float64 [V, H])."""
+    lib = _load()
+    code = _dtype_code(hidden)
+    assert _dtype_code(w) == code and hidden.ndim == 2 and w.ndim == 2 and hidden.shape[1] == w.shape[1]
+    assert hidden.strides[1] == hidden.itemsize and w.flags.c_contiguous
+    ids = np.ascontiguousarray(target_ids, dtype=np.int32)
+    g = np.ascontiguousarray(upstream, dtype=np.float64)
+    n, hdim = hidden.shape
+    assert ids.shape == (n,) and g.shape == (n,)
+    dh = np.empty((n, hdim), dtype=np.float64)
+    dw = np.empty((w.shape[0], hdim), dtype=np.float64) if want_dw else None
+    rc = lib.rpx_oracle_logprob_backward(_ptr(hidden), hidden.strides[0] // hidden.itemsize, _ptr(w), code, _ptr(ids),
+                                         _ptr(g), n, hdim, w.shape[0], _ptr(dh), _ptr(dw) if want_dw else None)
+    if rc != 0:
+        raise MemoryError(f"rpx_oracle_logprob_backward failed with {rc}")
+    return (dh, dw) if want_dw else dh
+
+
+def attn_backward(q, k, v, cu_seqlens, dout, scale=None):
+    """Gradients of sum(dout * O) for monolithic causal GQA attention over whole sequences (prompt then response).
+    q [T, H_q, d], k/v [T, H_kv, d] packed by cu_seqlens; dout float64 [T, H_q, d].
+    Returns (dq [T, H_q, d], dk [T, H_kv, d], dv [T, H_kv, d]) in float64."""
+    lib = _load()
+    code = _dtype_code(q)
+    assert _dtype_code(k) == code and _dtype_code(v) == code
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    hq, d = q.shape[1], q.shape[2]
+    hkv = k.shape[1]
+    total = int(cu[-1])
+    assert q.shape[0] == total and k.shape[0] == total and v.shape[0] == total
+    do = np.ascontiguousarray(dout, dtype=np.float64)
+    assert do.shape == (total, hq, d)
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    dq = np.empty((total, hq, d), dtype=np.float64)
+    dk = np.empty((total, hkv, d), dtype=np.float64)
+    dv = np.empty((total, hkv, d), dtype=np.float64)
+    rc = lib.rpx_oracle_attn_backward(_ptr(q), _ptr(k), _ptr(v), code, _tok_stride(q), _tok_stride(k), _tok_stride(v),
+                                      _ptr(cu), cu.shape[0] - 1, hq, hkv, d, float(scale), _ptr(do), _ptr(dq), _ptr(dk),
+                                      _ptr(dv))
+    if rc != 0:
+        raise ValueError(f"rpx_oracle_attn_backward failed with {rc}")
+    return dq, dk, dv

@@ -247,3 +247,177 @@ int rpx_oracle_cache_image(const void* k, const void* v, int dtype, int64_t k_to
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Backward through the boundary (Section 3.2, the autograd contract of the training actor's prefix; Table 4,
+ * row on the boundary prefix KV of the training actor, which stays attached to the graph): gradients of the
+ * suffix flow into the prefix through the retained K and V.  As in the forward direction the split is a
+ * re-ordering, so the oracle is the gradient of the monolithic definitions above, written out term by term.
+ *
+ *   LM head     with p_v = exp(z_v - lse) and an upstream gradient g[n] = dL / d logprob[n]:
+ *                   dL/dz_v      = g[n] * ([v == target] - p_v)
+ *                   dhidden[n,:] = sum_v dL/dz_v * W[v,:]
+ *                   dW[v,:]      = sum_n dL/dz_v(n) * hidden[n,:]
+ *   attention   with P_ij the softmax weights of row (i,h) over keys j <= i, g = h / (H_q / H_kv), and an
+ *               upstream gradient dO[i,h,:]:
+ *                   dP_ij = sum_c dO[i,h,c] * V[j,g,c]
+ *                   D_i   = sum_j P_ij * dP_ij
+ *                   dS_ij = P_ij * (dP_ij - D_i)
+ *                   dQ[i,h,:] = scale * sum_j dS_ij * K[j,g,:]
+ *                   dK[j,g,:] = scale * sum_{h in g} sum_{i >= j} dS_ij * Q[i,h,:]
+ *                   dV[j,g,:] =         sum_{h in g} sum_{i >= j} P_ij  * dO[i,h,:]
+ *               A key j of the prompt receives contributions from prompt queries and from response queries
+ *               alike: that sum over both is what "gradients flow from the suffix into the prefix" means.
+ * Pins (tests/test_oracle_backward_pins.py): central finite differences of the forward routines above,
+ * torch's fp64 autograd on CPU, closed forms (a one-key sequence, W = 0, uniform scores), the identity
+ * sum_v dL/dz_v = 0, and a split evaluation (prefix queries and suffix queries accumulated separately) against
+ * the monolithic sums.
+ */
+
+/*
+ * LM-head backward for all n rows.
+ *   upstream [n] (double), target_ids [n]; dhidden [n][hidden_dim] and dw [vocab][hidden_dim] (nullable) in double.
+ * A target outside [0, vocab) has no one-hot term (its log-prob is NaN in the forward pass); callers keep such rows
+ * out of the comparison.
+ */
+int rpx_oracle_logprob_backward(const void* hidden, int64_t hidden_row_stride, const void* w, int dtype,
+                                const int32_t* target_ids, const double* upstream, int64_t n, int32_t hidden_dim,
+                                int32_t vocab, double* dhidden, double* dw) {
+    double* dz = (double*)malloc(sizeof(double) * (size_t)n * (size_t)vocab);
+    if (!dz) return -2;
+    /* logits */
+#pragma omp parallel for schedule(static)
+    for (int32_t vv = 0; vv < vocab; ++vv) {
+        const int64_t woff = (int64_t)vv * hidden_dim;
+        for (int64_t r = 0; r < n; ++r) {
+            const int64_t hoff = r * hidden_row_stride;
+            double dot = 0.0;
+            for (int c = 0; c < hidden_dim; ++c)
+                dot += load_elem(hidden, dtype, hoff + c) * load_elem(w, dtype, woff + c);
+            dz[r * (int64_t)vocab + vv] = dot;
+        }
+    }
+    /* dL/dz = g * (onehot - softmax) */
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n; ++r) {
+        double* zr = dz + r * (int64_t)vocab;
+        double m = -INFINITY;
+        for (int32_t vv = 0; vv < vocab; ++vv)
+            if (zr[vv] > m) m = zr[vv];
+        double l = 0.0;
+        for (int32_t vv = 0; vv < vocab; ++vv) l += exp(zr[vv] - m);
+        const int32_t t = target_ids[r];
+        for (int32_t vv = 0; vv < vocab; ++vv) {
+            const double pv = exp(zr[vv] - m) / l;
+            zr[vv] = upstream[r] * ((vv == t ? 1.0 : 0.0) - pv);
+        }
+    }
+    /* dhidden = dz . W */
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n; ++r) {
+        double* dh = dhidden + r * (int64_t)hidden_dim;
+        for (int c = 0; c < hidden_dim; ++c) dh[c] = 0.0;
+        for (int32_t vv = 0; vv < vocab; ++vv) {
+            const double d = dz[r * (int64_t)vocab + vv];
+            const int64_t woff = (int64_t)vv * hidden_dim;
+            for (int c = 0; c < hidden_dim; ++c) dh[c] += d * load_elem(w, dtype, woff + c);
+        }
+    }
+    /* dW = dz^T . hidden */
+    if (dw) {
+#pragma omp parallel for schedule(static)
+        for (int32_t vv = 0; vv < vocab; ++vv) {
+            double* dwr = dw + (int64_t)vv * hidden_dim;
+            for (int c = 0; c < hidden_dim; ++c) dwr[c] = 0.0;
+            for (int64_t r = 0; r < n; ++r) {
+                const double d = dz[r * (int64_t)vocab + vv];
+                const int64_t hoff = r * hidden_row_stride;
+                for (int c = 0; c < hidden_dim; ++c) dwr[c] += d * load_elem(hidden, dtype, hoff + c);
+            }
+        }
+    }
+    free(dz);
+    return 0;
+}
+
+/*
+ * Monolithic causal GQA attention backward for whole sequences.
+ *   q, dout [tokens][H_q][d]; k, v [tokens][H_kv][d] (token strides in elements; dout is double, contiguous
+ *   [tokens][H_q][d]); dq [tokens][H_q][d], dk, dv [tokens][H_kv][d] in double, contiguous, written in full.
+ * Loops are over (sequence, head, query row), each row adding its terms into dk and dv of the keys it sees;
+ * rows of one KV head are taken by one thread, so no two threads add into the same element.
+ */
+int rpx_oracle_attn_backward(const void* q, const void* k, const void* v, int dtype, int64_t q_tok_stride,
+                             int64_t k_tok_stride, int64_t v_tok_stride, const int32_t* cu_seqlens, int32_t batch,
+                             int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, double scale,
+                             const double* dout, double* dq, double* dk, double* dv) {
+    if (num_kv_heads <= 0 || num_q_heads % num_kv_heads != 0) return -1;
+    const int group = num_q_heads / num_kv_heads;
+    const int64_t total = cu_seqlens[batch];
+    for (int64_t i = 0; i < total * num_q_heads * head_dim; ++i) dq[i] = 0.0;
+    for (int64_t i = 0; i < total * num_kv_heads * head_dim; ++i) dk[i] = dv[i] = 0.0;
+    int failed = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int32_t s = 0; s < batch; ++s) {
+        for (int32_t g = 0; g < num_kv_heads; ++g) {
+            const int64_t tok0 = cu_seqlens[s];
+            const int32_t len = cu_seqlens[s + 1] - cu_seqlens[s];
+            double* p = (double*)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+            double* dp = (double*)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+            if (!p || !dp) {
+#pragma omp atomic write
+                failed = 1;
+                free(p);
+                free(dp);
+                continue;
+            }
+            for (int32_t h = g * group; h < (g + 1) * group; ++h) {
+                for (int32_t i = 0; i < len; ++i) {
+                    const int64_t qoff = (tok0 + i) * q_tok_stride + (int64_t)h * head_dim;
+                    const double* dor = dout + ((tok0 + i) * num_q_heads + h) * head_dim;
+                    /* forward: P_ij */
+                    double m = -INFINITY;
+                    for (int32_t j = 0; j <= i; ++j) {
+                        const int64_t koff = (tok0 + j) * k_tok_stride + (int64_t)g * head_dim;
+                        double dot = 0.0;
+                        for (int c = 0; c < head_dim; ++c)
+                            dot += load_elem(q, dtype, qoff + c) * load_elem(k, dtype, koff + c);
+                        p[j] = dot * scale;
+                        if (p[j] > m) m = p[j];
+                    }
+                    double l = 0.0;
+                    for (int32_t j = 0; j <= i; ++j) {
+                        p[j] = exp(p[j] - m);
+                        l += p[j];
+                    }
+                    for (int32_t j = 0; j <= i; ++j) p[j] /= l;
+                    /* dP_ij and D_i */
+                    double big_d = 0.0;
+                    for (int32_t j = 0; j <= i; ++j) {
+                        const int64_t voff = (tok0 + j) * v_tok_stride + (int64_t)g * head_dim;
+                        double dot = 0.0;
+                        for (int c = 0; c < head_dim; ++c) dot += dor[c] * load_elem(v, dtype, voff + c);
+                        dp[j] = dot;
+                        big_d += p[j] * dot;
+                    }
+                    /* dS_ij, and the three gradients */
+                    double* dqr = dq + ((tok0 + i) * num_q_heads + h) * head_dim;
+                    for (int32_t j = 0; j <= i; ++j) {
+                        const double ds = p[j] * (dp[j] - big_d);
+                        const int64_t koff = (tok0 + j) * k_tok_stride + (int64_t)g * head_dim;
+                        double* dkr = dk + ((tok0 + j) * num_kv_heads + g) * head_dim;
+                        double* dvr = dv + ((tok0 + j) * num_kv_heads + g) * head_dim;
+                        for (int c = 0; c < head_dim; ++c) {
+                            dqr[c] += scale * ds * load_elem(k, dtype, koff + c);
+                            dkr[c] += scale * ds * load_elem(q, dtype, qoff + c);
+                            dvr[c] += p[j] * dor[c];
+                        }
+                    }
+                }
+            }
+            free(p);
+            free(dp);
+        }
+    }
+    return failed ? -2 : 0;
+}
