@@ -354,6 +354,59 @@ def measure_config(torch, dist, config, steps, warmup, rank, local_rank, world, 
     return rec
 
 
+def measure_backward(torch, config, local_rank, reps=3):
+    """The LM-head backward pass (dL/dz recomputed block by block from the saved lse, then dlogits x W) on the prompt
+    rows of one config: milliseconds, TFLOP/s on 4 * N * H * V algorithmic flops (the logits GEMM again plus the
+    dhidden GEMM), fractions of the measured peaks, and the clocks sampled meanwhile."""
+    import paper_2608_14498_b200 as rpx
+    from paper_2608_14498_b200 import binding as B
+
+    dev = torch.device("cuda", local_rank)
+    cfg = wk.CONFIGS[config]
+    wl = wk.make_workload(cfg, seed=0, attn=False)
+    pre = wl.prefix_rows()
+
+    def t(a):
+        x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return x.to(dev)
+
+    h, w, ids = t(wl.hidden[pre]), t(wl.w), t(wl.ids[pre])
+    n = h.shape[0]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    _, lse = rpx.token_logprobs(h, w, ids, return_lse=True, device_status=status)
+    g = torch.ones(n, dtype=torch.float32, device=dev)
+    dh = torch.empty_like(h)
+    ws = torch.empty(B.token_logprobs_backward_workspace_bytes(n, cfg.hidden, cfg.vocab), dtype=torch.uint8, device=dev)
+    rpx.token_logprobs_backward(h, w, ids, lse, g, dhidden=dh, workspace=ws, device_status=status)
+    torch.cuda.synchronize()
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(local_rank).uuid)
+        gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark()
+    e0.record()
+    for _ in range(reps):
+        rpx.token_logprobs_backward(h, w, ids, lse, g, dhidden=dh, workspace=ws, device_status=status)
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.mark()
+    clocks = sampler.stop()
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} in the backward pass")
+    ms = e0.elapsed_time(e1) / reps
+    peaks = load_peaks()
+    tf = 4.0 * n * cfg.hidden * cfg.vocab / (ms * 1e-3) / 1e12
+    return {"what": "rpx_token_logprobs_backward on the prompt rows (dL/dz from the saved lse, then dlogits x W)",
+            "workload": cfg.name, "rows": n, "ms": ms, "tflops": tf,
+            "frac_of_sustained_peak": tf / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+            "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]), "workspace_bytes": ws.numel(),
+            "gpu_launches": 2 * reps * -(-n // 9472), "clocks": clocks}
+
+
 def run_ours(args, rank, local_rank, world):
     import torch
     import torch.distributed as dist
@@ -380,6 +433,10 @@ def run_ours(args, rank, local_rank, world):
             others[name] = {k: sub[k] for k in ("value", "ms_per_step", "steps", "tflops", "frac_of_sustained_peak",
                                                 "frac_of_burst_peak", "kernels", "e2e", "clocks")}
             others[name]["workload"] = sub["config"]["workload"]
+    backward = None
+    if world == 1 and not args.no_backward:
+        torch.cuda.empty_cache()
+        backward = measure_backward(torch, "C2", local_rank)
     if rank == 0:
         line = {
             "metric": "scored_tokens_per_s", "value": head["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -389,6 +446,8 @@ def run_ours(args, rank, local_rank, world):
         line.update({k: v for k, v in head.items() if k not in ("value", "ms_per_step", "steps")})
         if others:
             line["configs"] = others
+        if backward:
+            line["backward"] = backward
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -511,6 +570,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="C3", choices=sorted(wk.CONFIGS), help="headline workload (C3 = the largest single-GPU config)")
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
+    ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
     ap.add_argument("--profile-case", choices=["lm", "prefix", "suffix"], help="launch one kernel a few times on a small case and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")

@@ -214,6 +214,31 @@ RPX_API rpx_status_t rpx_token_logprobs_merge(const float* shard_stats, int32_t 
                                               float* entropy, int32_t* device_status, void* cuda_stream);
 
 /*
+ * Backward of rpx_token_logprobs with respect to the hidden states (Section 3.2, the autograd contract of the
+ * training actor: its suffix and prefix passes are differentiated, and the gradient reaches the prefix through
+ * the retained boundary; Table 4, the row on the training actor's boundary KV, which stays attached).  The LM head is
+ * where that gradient starts.  With p = softmax(z[n,:]), z = hidden . w_vocab^T, and the caller's upstream gradient
+ * g[n] = dL / d logprobs[n]:
+ *     dL/dz[n,v]   = g[n] * ([v == target_ids[n]] - p_v)           (recomputed from lse, one block of rows at a time)
+ *     dhidden[n,:] = sum_v dL/dz[n,v] * w_vocab[v,:]
+ *   hidden, w_vocab, target_ids: as in the forward call; bf16 only (RPX_F32 returns RPX_ERR_DTYPE)
+ *   lse      device float32 [n_tokens]: the forward call's lse output for the same rows
+ *   upstream device float32 [n_tokens]
+ *   dhidden  bf16 [n_tokens][hidden_dim] contiguous, 16-byte aligned
+ *   workspace: rpx_token_logprobs_backward_workspace_bytes; it holds dL/dz of one block of at most 9472 rows as
+ *   bf16 (9472 x 152064 x 2 bytes = 2.9 GB for the 152064-column vocabulary), never of the whole batch.
+ * A target outside [0, vocab) contributes no one-hot term and sets RPX_ERR_DEVICE_DATA in *device_status.
+ * The weight gradient is not produced by this call.
+ */
+RPX_API rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                                 const int32_t* target_ids, const float* lse, const float* upstream,
+                                                 int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype,
+                                                 void* dhidden, void* workspace, size_t workspace_bytes,
+                                                 int32_t* device_status, void* cuda_stream);
+RPX_API size_t rpx_token_logprobs_backward_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                                           rpx_dtype_t dtype);
+
+/*
  * Allocation-free variant of rpx_token_logprobs (the paper has no counterpart: this entry point
  * exists for deployment, not for the method).  It is meant for callers that cannot give the
  * library a workspace because they cannot allocate one: a scoring hook that runs inside an

@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     suffix_attn,
     suffix_attn_workspace_bytes,
     token_logprobs,
+    token_logprobs_backward,
+    token_logprobs_backward_workspace_bytes,
     token_logprobs_merge,
     token_logprobs_shard,
     token_logprobs_static,

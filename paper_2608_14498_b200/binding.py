@@ -27,6 +27,8 @@ EXPORTS = (
     "rpx_token_logprobs_shard",
     "rpx_token_logprobs_merge",
     "rpx_token_logprobs_static",
+    "rpx_token_logprobs_backward",
+    "rpx_token_logprobs_backward_workspace_bytes",
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
     "rpx_token_logprobs_workspace_bytes",
@@ -100,6 +102,10 @@ def load_library():
     lib.rpx_token_logprobs_merge.argtypes = [vp, i32, vp, i64, i32, vp, vp, vp, vp, vp]
     lib.rpx_token_logprobs_static.restype = i32
     lib.rpx_token_logprobs_static.argtypes = [vp, i64, vp, vp, i64, i32, i32, vp, vp, vp, vp]
+    lib.rpx_token_logprobs_backward.restype = i32
+    lib.rpx_token_logprobs_backward.argtypes = [vp, i64, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_backward_workspace_bytes.restype = sz
+    lib.rpx_token_logprobs_backward_workspace_bytes.argtypes = [i64, i32, i32, i32]
     lib.rpx_prefix_attn_workspace_bytes.restype = sz
     lib.rpx_prefix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
     lib.rpx_suffix_attn_workspace_bytes.restype = sz
@@ -352,6 +358,38 @@ def token_logprobs(hidden, w_vocab, target_ids, logprobs=None, lse=None, return_
     if rc != 0:
         raise RpxError(rc, "rpx_token_logprobs")
     return (logprobs, lse) if return_lse else logprobs
+
+
+def token_logprobs_backward_workspace_bytes(n_tokens, hidden_dim, vocab, dtype_code=RPX_BF16) -> int:
+    return int(load_library().rpx_token_logprobs_backward_workspace_bytes(int(n_tokens), int(hidden_dim), int(vocab),
+                                                                          int(dtype_code)))
+
+
+@_in_call_context
+def token_logprobs_backward(hidden, w_vocab, target_ids, lse, upstream, dhidden=None, workspace=None, device_status=None,
+                            stream=None):
+    """rpx_token_logprobs_backward: d(sum upstream * logprobs) / d hidden, bf16 [N, H].
+
+    ``lse`` is the forward call's lse output for the same rows, ``upstream`` float32 [N]."""
+    torch = _torch()
+    lib = load_library()
+    if _dtype_code(hidden) != RPX_BF16 or _dtype_code(w_vocab) != RPX_BF16:
+        raise TypeError("the LM-head backward pass takes bfloat16 tensors only")
+    if hidden.dim() != 2 or hidden.stride(1) != 1 or not w_vocab.is_contiguous():
+        raise ValueError("hidden must be [N, H] with contiguous rows and w_vocab contiguous [V, H]")
+    if lse.dtype != torch.float32 or upstream.dtype != torch.float32:
+        raise TypeError("lse and upstream are float32")
+    n, hdim = hidden.shape
+    vocab = w_vocab.shape[0]
+    if dhidden is None:
+        dhidden = torch.empty((n, hdim), dtype=torch.bfloat16, device=hidden.device)
+    ws = _workspace(int(lib.rpx_token_logprobs_backward_workspace_bytes(n, hdim, vocab, RPX_BF16)), hidden.device, workspace)
+    rc = lib.rpx_token_logprobs_backward(_ptr(hidden), hidden.stride(0) if n > 1 else hdim, _ptr(w_vocab), _ptr(target_ids),
+                                         _ptr(lse), _ptr(upstream), n, hdim, vocab, RPX_BF16, _ptr(dhidden), _ptr(ws),
+                                         ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_token_logprobs_backward")
+    return dhidden
 
 
 @_in_call_context

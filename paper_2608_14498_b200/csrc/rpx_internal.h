@@ -75,6 +75,24 @@ rpx_status_t launch_logprob_merge(const void* shard_stats, int32_t n_shards, con
                                   int32_t vocab_total, float* logprobs, float* lse, float* entropy, int32_t* status,
                                   cudaStream_t stream);
 
+struct LogprobBwdArgs {
+    const void* hidden;        // bf16 [n][hidden_row_stride]
+    int64_t hidden_row_stride;
+    const void* w;             // bf16 [vocab][hidden_dim]
+    const int32_t* target_ids;
+    const float* lse;          // [n], from the forward call
+    const float* upstream;     // [n], dL / d logprob
+    int64_t n_tokens;
+    int32_t hidden_dim, vocab;
+    void* dhidden;             // bf16 [n][hidden_dim]
+    void* dlogits;             // workspace: bf16 [logprob_backward_block_rows(n)][vocab rounded up to 64]
+    int32_t* device_status;
+    cudaStream_t stream;
+};
+int64_t logprob_backward_block_rows(int64_t n_tokens);
+size_t logprob_backward_workspace(int64_t n_tokens, int32_t vocab);
+rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a);
+
 rpx_status_t launch_bounded_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t stream);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
