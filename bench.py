@@ -512,6 +512,9 @@ def run_group(args):
 
     dev = torch.device("cuda", 0)
     cfg = wk.CONFIGS[args.config]
+    if args.group_responses:  # e.g. 16:64 = response lengths uniform in [16, 64] (short answers: most of a query tile is padding)
+        lo, hi = (int(x) for x in args.group_responses.split(":"))
+        cfg = cfg.scaled(name=f"{cfg.name}-r{lo}to{hi}", response=("uniform", lo, hi))
     gw = wk.make_group_workload(cfg, args.group, seed=0)
     pro, mem = gw.prompts, gw.members
 
@@ -531,20 +534,25 @@ def run_group(args):
                      shared.cu_suffix, shared.prefix_lens, t(own_table), t(mem.hidden[pre]), t(mem.ids[pre]), shared.hidden_s,
                      shared.ids_s, shared.max_prefix_len, shared.max_suffix_len)
 
-    def timed(session, batch):
+    def timed(session, batch, kernel_ms=None):
         for _ in range(3):
             session.score(batch)
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            session.score(batch)
-        e1.record()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+        for s in range(args.steps):
+            session.score(batch, events=ev[s])
         torch.cuda.synchronize()
         session.check_status()
-        return e0.elapsed_time(e1) / args.steps
+        if kernel_ms is not None:
+            for i, n in enumerate(["prefix_attn", "lm_prefix", "suffix_attn", "lm_suffix"]):
+                kernel_ms[n] = sum(e[i].elapsed_time(e[i + 1]) for e in ev) / args.steps
+        return ev[0][0].elapsed_time(ev[-1][4]) / args.steps
 
-    ms_shared, ms_unshared = timed(sess, shared), timed(sess_own, unshared)
+    kernel_ms = {}
+    ms_shared, ms_unshared = timed(sess, shared, kernel_ms), timed(sess_own, unshared)
+    r = mem.response_lens.astype(np.float64)
+    pl = mem.prompt_lens.astype(np.float64)
+    suffix_flops = float((4.0 * cfg.head_dim * cfg.num_q_heads * (r * pl + r * (r + 1) / 2)).sum())
     lp_a = sess.score(shared)[1].clone()
     lp_b = sess_own.score(unshared)[1]
     torch.cuda.synchronize()
@@ -553,7 +561,10 @@ def run_group(args):
         "steps": args.steps, "warmup": 3, "ms_per_step": ms_shared, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{cfg.name} as {cfg.batch} prompts x {args.group} responses, prefix scored once per prompt",
-                   "member_tokens": mem.n_tokens, "prompt_rows_computed": pro.n_tokens, "response_rows": mem.n_suffix},
+                   "member_tokens": mem.n_tokens, "prompt_rows_computed": pro.n_tokens, "response_rows": mem.n_suffix,
+                   "response_lens": [int(mem.response_lens.min()), int(mem.response_lens.max())]},
+        "kernels_ms": {k: round(v, 4) for k, v in kernel_ms.items()},
+        "suffix_attn_tflops": suffix_flops / (kernel_ms["suffix_attn"] * 1e-3) / 1e12,
         "group": {"size": args.group, "ms_shared_prefix": ms_shared, "ms_every_member_own_prefix": ms_unshared,
                   "speedup": ms_unshared / ms_shared,
                   "suffix_logprob_max_abs_diff": float((lp_a - lp_b).abs().max().item())},
@@ -577,6 +588,7 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--group", type=int, default=0, help="score prompt groups of this size (prefix once per prompt)")
+    ap.add_argument("--group-responses", default="", help="with --group: LO:HI = response lengths uniform in [LO, HI]")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -90,6 +90,13 @@ struct Params {
     int32_t write_cache;          // store this call's K/V into the cache (prefix pass, chunked prefill)
     int32_t batch, num_q_heads, num_kv_heads, group;
     int32_t n_pairs;              // query tile pairs per sequence the work list covers
+    // Row packing (suffix pass): a query tile holds tile_tokens = 128 / group consecutive tokens times the `group`
+    // query heads of ONE KV head (row = token * group + head within the group), so a cached K/V tile is fetched once
+    // per KV head instead of once per query head and a short response fills its tile.  pack == 0: a tile is 128
+    // tokens of one query head.
+    int32_t pack;
+    int32_t tile_tokens;          // query tokens per tile: 128, or 128 / group when packed
+    int32_t item_heads;           // heads the work list runs over: num_q_heads, or num_kv_heads when packed
     int32_t n_items;              // n_pairs * batch * num_q_heads
     uint32_t* next_item;          // device counter, zero before the launch: work items are handed out in order
     // Split-KV (suffix passes with few, long items): the cached prefix of an item is cut into n_splits
@@ -118,7 +125,7 @@ __device__ __forceinline__ uint32_t swz_off(int r, int cc) {
 struct Item {
     int32_t pair, seq, head, kv_head, tok0, len_q, q0, len_p, n_prefix_tiles, n_tile0, n_kv;
     int32_t pt0;      // first cached tile this item walks (n_prefix_tiles counts the tiles of its range)
-    int32_t x1;       // extra key steps of query tile 1 over tile 0: 1 when the item holds the self tiles, else 0
+    int32_t x1;       // extra key steps of query tile 1 over tile 0 (0 or 1)
     int32_t split, s_eff;  // which range of the cached prefix, out of how many (1 = the whole item)
     bool active, active1;
 };
@@ -129,7 +136,7 @@ struct Item {
 // negative cached length, more pages than a row of the block table holds) are reported and the item is handed on
 // empty, so nothing is read or written through them.
 __device__ __forceinline__ int4 fetch_item(const Params& p, int32_t idx, uint32_t* data_error) {
-    const int32_t seq = ((idx / p.n_splits) % (p.batch * p.num_q_heads)) / p.num_q_heads;
+    const int32_t seq = ((idx / p.n_splits) % (p.batch * p.item_heads)) / p.item_heads;
     const int32_t tok0 = __ldg(p.cu_seqlens + seq);
     int32_t len_q = __ldg(p.cu_seqlens + seq + 1) - tok0;
     int32_t len_p = p.prefix_lens != nullptr ? __ldg(p.prefix_lens + seq) : 0;
@@ -153,29 +160,34 @@ __device__ __forceinline__ Item decode_item(const Params& p, int4 rec) {
     Item it;
     const int32_t idx = rec.x / p.n_splits;  // the item's (pair, sequence, head); its splits are numbered consecutively
     it.split = rec.x % p.n_splits;
-    const int32_t per_pair = p.batch * p.num_q_heads;
+    const int32_t per_pair = p.batch * p.item_heads;
     it.pair = p.n_pairs - 1 - idx / per_pair;
     const int32_t rem = idx % per_pair;
-    it.seq = rem / p.num_q_heads;
-    it.head = rem % p.num_q_heads;
-    it.kv_head = it.head / p.group;
+    it.seq = rem / p.item_heads;
+    it.head = rem % p.item_heads;  // packed: the KV head whose query heads share the tile
+    it.kv_head = p.pack != 0 ? it.head : it.head / p.group;
     it.tok0 = rec.y;
     it.len_q = rec.z;
-    it.q0 = it.pair * 2 * kTileQ;
+    it.q0 = it.pair * 2 * p.tile_tokens;
     it.active = it.q0 < it.len_q;
     it.len_p = it.active ? rec.w : 0;
-    it.active1 = it.q0 + kTileQ < it.len_q;
+    it.active1 = it.q0 + p.tile_tokens < it.len_q;
     const int32_t n_pt = (it.len_p + kTileK - 1) / kTileK;  // cached tiles of the whole prefix
     it.s_eff = max(1, min(p.n_splits, n_pt));                // a prefix shorter than n_splits tiles is cut in fewer
     if (it.split >= it.s_eff) it.active = false;
     it.pt0 = n_pt * min(it.split, it.s_eff) / it.s_eff;
     it.n_prefix_tiles = n_pt * min(it.split + 1, it.s_eff) / it.s_eff - it.pt0;
-    it.x1 = it.split == it.s_eff - 1 ? 1 : 0;                // the last range also takes the self tiles
+    // self key tiles each query tile walks: up to the tile that holds its last token (the last range of a split
+    // item takes them, the others none)
+    const int32_t last = it.split == it.s_eff - 1 ? 1 : 0;
+    const int32_t self0 = (min(it.len_q, it.q0 + p.tile_tokens) + kTileK - 1) / kTileK;
+    const int32_t self1 = it.active1 ? (min(it.len_q, it.q0 + 2 * p.tile_tokens) + kTileK - 1) / kTileK : self0;
     // key steps of query tile t: n_tile0 + t * x1.  (Scalars, not arrays: a small array indexed at
     // run time lives in local memory, and with nearly all L1 carved out as shared memory every such
     // load stalls the in-order warp for hundreds of cycles.)
-    it.n_tile0 = it.n_prefix_tiles + it.x1 * (2 * it.pair + 1);
-    it.n_kv = it.n_tile0 + (it.active1 ? it.x1 : 0);
+    it.n_tile0 = it.n_prefix_tiles + last * self0;
+    it.x1 = last * (self1 - self0);  // 0 or 1: a tile spans at most 128 tokens
+    it.n_kv = it.n_tile0 + it.x1;
     return it;
 }
 
@@ -274,7 +286,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             if (rec.x < 0) break;
             const Item it = decode_item(p, rec);
             // A sequence longer than the caller's bound would leave rows the work list never reaches: report it.
-            if (it.pair == 0 && it.head == 0 && lane == 0 && it.len_q > p.n_pairs * 2 * kTileQ) ctl->data_error = 1;
+            if (it.pair == 0 && it.head == 0 && lane == 0 && it.len_q > p.n_pairs * 2 * p.tile_tokens) ctl->data_error = 1;
             if (!it.active) continue;
             const int32_t pair = it.pair, seq = it.seq, head = it.head, kv_head = it.kv_head, tok0 = it.tok0;
             const int32_t len_q = it.len_q, q0 = it.q0, len_p = it.len_p, n_prefix_tiles = it.n_prefix_tiles;
@@ -288,17 +300,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 break;
             }
             if (lane == 0) {
-            mbar_arrive_expect_tx(&ctl->q_full, (active1 ? 2 : 1) * L::kQBytes);
-            for (int t = 0; t < (active1 ? 2 : 1); ++t)
-                for (int hf = 0; hf < L::kHalves; ++hf)
-                    tma_load_3d(smem + L::kQOff + t * L::kQBytes + hf * L::kHalfBytes, &tmap_q, &ctl->q_full,
-                                hf * 64, head, tok0 + q0 + t * kTileQ);
-        }
+                // packed: one box of tile_tokens tokens x group heads lands as consecutive 128-byte rows (token-major)
+                const int32_t rows = p.pack != 0 ? p.tile_tokens * p.group : kTileQ;
+                mbar_arrive_expect_tx(&ctl->q_full, (active1 ? 2 : 1) * L::kHalves * rows * 128);
+                for (int t = 0; t < (active1 ? 2 : 1); ++t)
+                    for (int hf = 0; hf < L::kHalves; ++hf)
+                        tma_load_3d(smem + L::kQOff + t * L::kQBytes + hf * L::kHalfBytes, &tmap_q, &ctl->q_full, hf * 64,
+                                    p.pack != 0 ? kv_head * p.group : head, tok0 + q0 + t * p.tile_tokens);
+            }
         // Appending behind a cached prefix (chunked prefill) needs the chunk to start on a page edge:
         // pages are written whole or from their first row.  Anything else is reported, not written.
         const bool page_aligned = (len_p % kPage) == 0;
         if (p.write_cache != 0 && !page_aligned && lane == 0) ctl->data_error = 1;
-        const bool owns_cache_write = p.write_cache != 0 && page_aligned && (head % p.group) == 0;
+        const bool owns_cache_write = p.write_cache != 0 && p.pack == 0 && page_aligned && (head % p.group) == 0;
         const int32_t write_page0 = len_p / kPage;  // first page of this call's own tokens
         // Block id of page `lane` of cached tile jt (lanes 0..7; 0 where the prefix has no such page).
         // Read one tile ahead, so the table's global-memory latency is off the ring's critical path.
@@ -477,7 +491,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // 16 keys of P = 8 TMEM columns of packed bf16 pairs; 16 keys of V = 2 KiB of rows
                 const uint64_t vd = v_desc0 + static_cast<uint64_t>(v_slot * (L::kKvBytes >> 4));
                 umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128, vd, idesc_pv, accumulate ? 1u : 0u);
-                if (it.s_eff == 1 && n_tile0 + t <= 2)  // + P_lo V, P_lo in columns 64..127 of S_t
+                if (it.s_eff == 1 && n_tile0 + t * x1 <= 2)  // + P_lo V, P_lo in columns 64..127 of S_t
                     umma_ts_k128(tmem_base + 256 + t * 128, tmem_base + t * 128 + 64, vd, idesc_pv, 1u);
             };
 
@@ -569,7 +583,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             (void)n_prefix_tiles; (void)n_tile0; (void)n_kv; (void)active1; (void)pt0; (void)x1;
             const uint32_t quarter = warp & 3;
             const int32_t row = quarter * 32 + lane;
-            const int32_t q_local = q0 + t * kTileQ + row;  // position among this call's query tokens
+            // which query token and head this thread's row is: unpacked, row = token of the item's head; packed,
+            // row = token * group + head within the KV head's group (rows beyond tile_tokens * group are padding)
+            int32_t q_local, row_head;  // position among this call's query tokens; query head
+            bool row_in_tile = true;
+            if (p.pack != 0) {
+                const int32_t tok = row / p.group;
+                q_local = q0 + t * p.tile_tokens + tok;
+                row_head = kv_head * p.group + (row - tok * p.group);
+                row_in_tile = tok < p.tile_tokens;
+            } else {
+                q_local = q0 + t * kTileQ + row;
+                row_head = head;
+            }
             const uint32_t lane_addr = (quarter * 32u) << 16;
             const int32_t my_tiles = n_tile0 + t * x1;
             const uint32_t my_s = tmem_base + t * 128 + lane_addr;        // this thread's lane of S_t / P_t
@@ -725,9 +751,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             ++items_t;
             if (ok) {
                 tc_fence_after_sync();
-                const bool row_valid = q_local < len_q;
+                const bool row_valid = row_in_tile && q_local < len_q;
                 float inv = 1.f / run_sum;
-                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head) * D;
+                const int64_t out_row = (static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + row_head) * D;
                 // two chunks of 32 columns in flight: the next chunk's TMEM load runs under this chunk's stores
                 uint32_t ra[32], rb[32];
                 // A warp's store instruction touches 32 rows, so its cost is the number of 32-byte sectors
@@ -770,7 +796,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 if (it.s_eff > 1) {
                     // ---- one range of a split item: the un-normalised row and its (maximum, sum) go to the
                     // workspace; whichever of the s_eff CTAs arrives last for these 32 rows merges them
-                    const int64_t rh = static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head;
+                    const int64_t rh = static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + row_head;
                     const int64_t per_split = p.total_tokens * p.num_q_heads;
                     float* po = p.part_o + (static_cast<int64_t>(it.split) * per_split + rh) * D;
 #pragma unroll 1
@@ -789,15 +815,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                                              ra[8 * i + 4], ra[8 * i + 5], ra[8 * i + 6], ra[8 * i + 7]);
                         }
                     }
-                    const bool warp_valid = q0 + t * kTileQ + static_cast<int32_t>(quarter) * 32 < len_q;  // lane 0's row
+                    // rows are ordered by token, so when lane 0's row is beyond the sequence the whole warp's are
+                    const bool warp_valid = __shfl_sync(0xffffffffu, row_valid ? 1 : 0, 0) != 0;
                     if (row_valid) p.part_ml[static_cast<int64_t>(it.split) * per_split + rh] = make_float2(run_max, run_sum);
                     uint32_t arrived = 0;
+                    const int64_t rh_lane0 = __shfl_sync(0xffffffffu, rh, 0);  // the 32-row group's arrival counter
                     if (warp_valid) {
                         __threadfence();
                         __syncwarp();
-                        if (lane == 0)
-                            arrived = atomicAdd(p.split_cnt + (static_cast<int64_t>(tok0 + q0 + t * kTileQ) + quarter * 32) *
-                                                                  p.num_q_heads + head, 1u);
+                        if (lane == 0) arrived = atomicAdd(p.split_cnt + rh_lane0, 1u);
                         arrived = __shfl_sync(0xffffffffu, arrived, 0);
                     }
                     if (warp_valid && arrived == static_cast<uint32_t>(it.s_eff - 1)) {
@@ -865,7 +891,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     store_chunk(rb, c + 1);
                 }
                 if (row_valid && p.lse != nullptr)
-                    p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + head] = (run_max + log2f(run_sum)) * kLn2;
+                    p.lse[static_cast<int64_t>(tok0 + q_local) * p.num_q_heads + row_head] = (run_max + log2f(run_sum)) * kLn2;
                 }
             }
         }
@@ -888,10 +914,15 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     using L = Layout<D>;
     CUtensorMap tq, tk, tv, tkc, tvc;
     const uint64_t tokens = static_cast<uint64_t>(a.total_tokens);
+    // Row packing: in the suffix pass the query heads of one KV head share a tile (see Params::pack).  Not for passes
+    // that store K/V (one writer per KV head is chosen among the per-head items) and pointless without grouping.
+    const int32_t group = a.num_q_heads / a.num_kv_heads;
+    const bool pack = a.prefix_lens != nullptr && !(a.cache != nullptr && a.append_cache) && group >= 2 && group <= kTileQ;
+    const int32_t tile_tokens = pack ? kTileQ / group : kTileQ;
     {
         const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_q_heads), tokens};
         const uint64_t strides[2] = {D * 2ull, static_cast<uint64_t>(a.q_tok_stride) * 2};
-        const uint32_t box[3] = {64, 1, kTileQ};
+        const uint32_t box[3] = {64, pack ? static_cast<uint32_t>(group) : 1u, static_cast<uint32_t>(tile_tokens)};
         if (rpx_status_t rc = encode_tmap_bf16(&tq, a.q, 3, dims, strides, box)) return rc;
     }
     {
@@ -924,8 +955,11 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.batch = a.batch;
     p.num_q_heads = a.num_q_heads;
     p.num_kv_heads = a.num_kv_heads;
-    p.group = a.num_q_heads / a.num_kv_heads;
-    p.n_pairs = (a.max_q_len + 2 * kTileQ - 1) / (2 * kTileQ);
+    p.group = group;
+    p.pack = pack ? 1 : 0;
+    p.tile_tokens = tile_tokens;
+    p.item_heads = pack ? a.num_kv_heads : a.num_q_heads;
+    p.n_pairs = (a.max_q_len + 2 * tile_tokens - 1) / (2 * tile_tokens);
     const float scale = a.softmax_scale > 0.f ? a.softmax_scale : 1.0f / sqrtf(static_cast<float>(D));
     p.scale_log2 = scale * kLog2e;
     p.inv_scale_log2 = 1.0f / p.scale_log2;
@@ -933,7 +967,7 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.out_f32 = a.out_f32 ? 1 : 0;
     p.lse = a.lse;
     p.status = a.device_status;
-    const int64_t n_base = static_cast<int64_t>(p.n_pairs) * a.batch * a.num_q_heads;
+    const int64_t n_base = static_cast<int64_t>(p.n_pairs) * a.batch * p.item_heads;
     if (n_base <= 0) return RPX_OK;
     int sms_all = sm_count();
     if (sms_all <= 0) return RPX_ERR_CUDA;
@@ -949,7 +983,7 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     if (a.prefix_lens != nullptr && p.write_cache == 0 && a.split_ws != nullptr &&
         attn_split_workspace(a.total_tokens, a.num_q_heads, D) > 0) {
         const int64_t prefix_steps = (a.max_prefix_len + kTileK - 1) / kTileK;
-        const int64_t self_steps = 2 * p.n_pairs + 1;
+        const int64_t self_steps = (static_cast<int64_t>(a.max_q_len) + kTileK - 1) / kTileK;
         // rounds of items x (key steps + about four steps' worth of fixed cost per item); with three ranges on C2's
         // suffix pass (224 items of 35 steps) the merge and the fixed costs ate the gain: 0.219 against 0.156 ms
         auto cost = [&](int64_t S) { return ((n_base * S + sms_all - 1) / sms_all) * (prefix_steps / S + 4) + self_steps; };
