@@ -2,7 +2,7 @@
 """Benchmark of the prefix+suffix scoring hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3]
-    python bench.py --profile-case lm|prefix|suffix [--reps 3]      (small launches for profiler captures)
+    python bench.py --profile-case lm|lmbwd|prefix|suffix [--reps 3]      (small launches for profiler captures)
 
 One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
 boundary-KV write), prefix log-probs, suffix attention over the cached KV, suffix log-probs.
@@ -46,7 +46,7 @@ from paper_2608_14498_b200 import workloads as wk  # noqa: E402
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the LM-head partial kernel on a config's
 # prompt rows, from one-pass ncu captures of this very command on that config.  Configs without a capture: None.
-LM_HEAD_TRAFFIC_BYTES = {"C2": 13.291e9 + 43.8e6}
+LM_HEAD_TRAFFIC_BYTES = {"C2": 13.291e9 + 43.8e6, "C3": 321.94e9 + 264.6e6}
 
 
 def load_peaks():
@@ -459,6 +459,7 @@ def run_profile_case(args):
     the device (more than the 126 MB L2, so DRAM counters mean something) and launches the kernel `reps` times
     after one warm-up launch.
       lm      8192 rows x 32768 vocabulary columns, hidden 3584  (7B-shaped slice of the LM head)
+      lmbwd   the same slice through rpx_token_logprobs_backward (two kernels per launch: dL/dz, then dhidden)
       prefix  4 sequences x 4096 prompt tokens, 28 query / 4 KV heads, head_dim 128, with cache write
       suffix  the same 4 prompts cached, 256 response tokens each"""
     import torch
@@ -480,6 +481,14 @@ def run_profile_case(args):
         h, w, ids = dv(wl.hidden), dv(wl.w), dv(wl.ids)
         for _ in range(1 + args.reps):
             rpx.token_logprobs(h, w, ids, device_status=status)
+    elif case == "lmbwd":
+        cfg = wk.Config("profile-lm", "bf16", 1, 28, 4, 128, 3584, 32768, ("fixed", 8192), ("fixed", 0))
+        wl = wk.make_workload(cfg, seed=0, attn=False)
+        h, w, ids = dv(wl.hidden), dv(wl.w), dv(wl.ids)
+        _, lse = rpx.token_logprobs(h, w, ids, return_lse=True, device_status=status)
+        g = torch.ones(h.shape[0], dtype=torch.float32, device=dev)
+        for _ in range(1 + args.reps):
+            rpx.token_logprobs_backward(h, w, ids, lse, g, device_status=status)
     else:
         cfg = wk.Config("profile-attn", "bf16", 4, 28, 4, 128, 3584, 1024, ("fixed", 4096), ("fixed", 256))
         wl = wk.make_workload(cfg, seed=0, lm=False)
@@ -582,7 +591,7 @@ def main():
     ap.add_argument("--config", default="C3", choices=sorted(wk.CONFIGS), help="headline workload (C3 = the largest single-GPU config)")
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
     ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
-    ap.add_argument("--profile-case", choices=["lm", "prefix", "suffix"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix"], help="launch one kernel a few times on a small case and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
