@@ -239,6 +239,41 @@ RPX_API size_t rpx_token_logprobs_backward_workspace_bytes(int64_t n_tokens, int
                                                            rpx_dtype_t dtype);
 
 /*
+ * Backward of causal GQA attention over packed whole sequences (Section 3.2: the training actor differentiates both
+ * its suffix pass and its prefix pass, and the suffix pass's gradient reaches the prompt through the prefix K/V it
+ * attended to; Table 4, the row on the boundary KV that stays attached).  A sequence is prompt followed by response;
+ * with P the softmax weights of query row (i, h) over the keys j <= i of its sequence (recomputed from lse), g the KV
+ * head of h, dP_ij = dout[i,h,:] . v[j,g,:], D_i = sum_c dout[i,h,c] * out[i,h,c] and dS_ij = P_ij (dP_ij - D_i):
+ *     dv[j,g,:] = sum_{h in g} sum_{i >= j} P_ij  dout[i,h,:]
+ *     dk[j,g,:] = scale * sum_{h in g} sum_{i >= j} dS_ij q[i,h,:]
+ *     dq[i,h,:] = scale * sum_{j <= i} dS_ij k[j,g,:]
+ *   q, k, v, strides, cu_seqlens, batch, total_tokens, max_seqlen: as in rpx_prefix_attn; bf16 only (RPX_F32
+ *       returns RPX_ERR_DTYPE)
+ *   out, dout  device bf16 [total_tokens][num_q_heads][head_dim] contiguous: the forward output and its gradient
+ *   lse        device float32 [total_tokens][num_q_heads]: the forward pass's lse (natural log)
+ *   q_begin, q_end   nullable device int32 [batch]: only the query rows q_begin[s] <= i < q_end[s] of sequence s take
+ *       part (clamped to the sequence; NULL = 0 and the sequence length).  Rows outside get dq = 0 and add nothing
+ *       to dk, dv.  With q_begin = prompt length the call is the suffix pass's backward (the gradient of the
+ *       response rows with respect to their own K/V and to the prompt's K/V); with q_end = prompt length it is
+ *       the prefix pass's.
+ *   dq         device float32 [total_tokens][num_q_heads][head_dim], written (rows outside the range: 0)
+ *   dk, dv     device float32 [total_tokens][num_kv_heads][head_dim]; accumulate_dkv == 0: written;
+ *       != 0: the call's dk, dv are ADDED to what the buffers hold, so that the suffix pass's call followed by the
+ *       prefix pass's call leaves the same sums as one call over all rows
+ *   workspace: rpx_attn_backward_workspace_bytes (D, 4 bytes per token and query head), 256-byte aligned
+ * P and dS are rounded to bf16 before they enter the tensor-core products, as P is in the forward pass.
+ * cu_seqlens that leave the packed tensors are not followed and set RPX_ERR_DEVICE_DATA in *device_status.
+ */
+RPX_API rpx_status_t rpx_attn_backward(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                                       int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const void* out,
+                                       const void* dout, const float* lse, const int32_t* cu_seqlens,
+                                       const int32_t* q_begin, const int32_t* q_end, int32_t batch, int64_t total_tokens,
+                                       int32_t max_seqlen, float* dq, float* dk, float* dv, int32_t accumulate_dkv,
+                                       void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                       void* cuda_stream);
+RPX_API size_t rpx_attn_backward_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens);
+
+/*
  * Allocation-free variant of rpx_token_logprobs (the paper has no counterpart: this entry point
  * exists for deployment, not for the method).  It is meant for callers that cannot give the
  * library a workspace because they cannot allocate one: a scoring hook that runs inside an

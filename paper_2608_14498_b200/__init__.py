@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     suffix_attn,
     suffix_attn_workspace_bytes,
     token_logprobs,
+    attn_backward,
     token_logprobs_backward,
     token_logprobs_backward_workspace_bytes,
     token_logprobs_merge,

@@ -29,6 +29,8 @@ EXPORTS = (
     "rpx_token_logprobs_static",
     "rpx_token_logprobs_backward",
     "rpx_token_logprobs_backward_workspace_bytes",
+    "rpx_attn_backward",
+    "rpx_attn_backward_workspace_bytes",
     "rpx_prefix_attn_workspace_bytes",
     "rpx_suffix_attn_workspace_bytes",
     "rpx_token_logprobs_workspace_bytes",
@@ -106,6 +108,11 @@ def load_library():
     lib.rpx_token_logprobs_backward.argtypes = [vp, i64, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, sz, vp, vp]
     lib.rpx_token_logprobs_backward_workspace_bytes.restype = sz
     lib.rpx_token_logprobs_backward_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    lib.rpx_attn_backward.restype = i32
+    lib.rpx_attn_backward.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, i32,
+                                      i64, i32, vp, vp, vp, i32, vp, sz, vp, vp]
+    lib.rpx_attn_backward_workspace_bytes.restype = sz
+    lib.rpx_attn_backward_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
     lib.rpx_prefix_attn_workspace_bytes.restype = sz
     lib.rpx_prefix_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), i64]
     lib.rpx_suffix_attn_workspace_bytes.restype = sz
@@ -390,6 +397,44 @@ def token_logprobs_backward(hidden, w_vocab, target_ids, lse, upstream, dhidden=
     if rc != 0:
         raise RpxError(rc, "rpx_token_logprobs_backward")
     return dhidden
+
+
+@_in_call_context
+def attn_backward(q, k, v, out, dout, lse, cu_seqlens, max_seqlen: int, q_begin=None, q_end=None, softmax_scale: float = 0.0,
+                  dq=None, dk=None, dv=None, accumulate_dkv: bool = False, workspace=None, device_status=None, stream=None):
+    """rpx_attn_backward: gradients of causal GQA attention over packed whole sequences.
+
+    q [T, H_q, d], k/v [T, H_kv, d], out/dout [T, H_q, d] bfloat16; lse float32 [T, H_q] from the forward pass;
+    q_begin / q_end (int32 [B], optional) restrict the query rows that take part.  Returns float32 (dq, dk, dv);
+    with ``accumulate_dkv`` the call's dk, dv are added to the given buffers."""
+    torch = _torch()
+    lib = load_library()
+    if any(_dtype_code(t) != RPX_BF16 for t in (q, k, v, out, dout)):
+        raise TypeError("the attention backward pass takes bfloat16 tensors only")
+    if lse.dtype != torch.float32 or not lse.is_contiguous() or not out.is_contiguous() or not dout.is_contiguous():
+        raise ValueError("out, dout and lse (float32) must be contiguous")
+    desc = _desc(q, k, softmax_scale)
+    total = q.shape[0]
+    if dq is None:
+        dq = torch.empty(tuple(q.shape), dtype=torch.float32, device=q.device)
+    if accumulate_dkv and (dk is None or dv is None):
+        raise ValueError("accumulate_dkv needs the dk and dv buffers to add to")
+    if dk is None:
+        dk = torch.empty(tuple(k.shape), dtype=torch.float32, device=q.device)
+    if dv is None:
+        dv = torch.empty(tuple(v.shape), dtype=torch.float32, device=q.device)
+    for t in (dq, dk, dv):
+        if t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError("dq, dk, dv are contiguous float32 tensors")
+    ws = _workspace(int(lib.rpx_attn_backward_workspace_bytes(ctypes.byref(desc), total)), q.device, workspace)
+    rc = lib.rpx_attn_backward(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _tok_stride(q), _tok_stride(k),
+                               _tok_stride(v), _ptr(out), _ptr(dout), _ptr(lse), _ptr(cu_seqlens), _ptr(q_begin),
+                               _ptr(q_end), cu_seqlens.shape[0] - 1, total, int(max_seqlen), _ptr(dq), _ptr(dk), _ptr(dv),
+                               1 if accumulate_dkv else 0, _ptr(ws), ws.numel() * ws.element_size(), _ptr(device_status),
+                               _stream_ptr(stream))
+    if rc != 0:
+        raise RpxError(rc, "rpx_attn_backward")
+    return dq, dk, dv
 
 
 @_in_call_context

@@ -316,6 +316,65 @@ rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_
     return launch_token_logprobs_backward(a);
 }
 
+size_t rpx_attn_backward_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens) {
+    if (desc == nullptr || total_tokens <= 0 || desc->num_q_heads <= 0) return 0;
+    return align_up(static_cast<size_t>(total_tokens) * desc->num_q_heads * sizeof(float), kWsAlign);
+}
+
+rpx_status_t rpx_attn_backward(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
+                               int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const void* out,
+                               const void* dout, const float* lse, const int32_t* cu_seqlens, const int32_t* q_begin,
+                               const int32_t* q_end, int32_t batch, int64_t total_tokens, int32_t max_seqlen, float* dq,
+                               float* dk, float* dv, int32_t accumulate_dkv, void* workspace, size_t workspace_bytes,
+                               int32_t* device_status, void* cuda_stream) {
+    if (rpx_status_t rc = check_attn_desc(desc)) return rc;
+    if (desc->dtype != RPX_BF16) return RPX_ERR_DTYPE;  // the backward pass takes bf16 tensors only
+    if (batch < 0 || total_tokens < 0 || max_seqlen < 0 || total_tokens >= INT32_MAX) return RPX_ERR_SHAPE;
+    if (batch == 0 || total_tokens == 0 || max_seqlen == 0) return RPX_OK;
+    if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || dout == nullptr || lse == nullptr ||
+        cu_seqlens == nullptr || dq == nullptr || dk == nullptr || dv == nullptr)
+        return RPX_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return RPX_ERR_ALIGN;
+    const int64_t q_row = static_cast<int64_t>(desc->num_q_heads) * desc->head_dim;
+    const int64_t kv_row = static_cast<int64_t>(desc->num_kv_heads) * desc->head_dim;
+    if (q_tok_stride < q_row || k_tok_stride < kv_row || v_tok_stride < kv_row) return RPX_ERR_SHAPE;
+    if (q_tok_stride % 8 || k_tok_stride % 8 || v_tok_stride % 8) return RPX_ERR_ALIGN;
+    const size_t need = rpx_attn_backward_workspace_bytes(desc, total_tokens);
+    if (workspace == nullptr || workspace_bytes < need) return RPX_ERR_WORKSPACE;
+    if (!aligned_ws(workspace)) return RPX_ERR_ALIGN;
+    if (rpx_status_t rc = check_arch()) return rc;
+    AttnBwdArgs a;
+    a.num_q_heads = desc->num_q_heads;
+    a.num_kv_heads = desc->num_kv_heads;
+    a.head_dim = desc->head_dim;
+    a.softmax_scale = desc->softmax_scale;
+    a.q = q;
+    a.k = k;
+    a.v = v;
+    a.q_tok_stride = q_tok_stride;
+    a.k_tok_stride = k_tok_stride;
+    a.v_tok_stride = v_tok_stride;
+    a.out = out;
+    a.dout = dout;
+    a.lse = lse;
+    a.cu_seqlens = cu_seqlens;
+    a.q_begin = q_begin;
+    a.q_end = q_end;
+    a.batch = batch;
+    a.total_tokens = total_tokens;
+    a.max_seqlen = max_seqlen;
+    a.dq = dq;
+    a.dk = dk;
+    a.dv = dv;
+    a.accumulate = accumulate_dkv != 0;
+    a.dvec = static_cast<float*>(workspace);
+    a.device_status = device_status;
+    a.stream = static_cast<cudaStream_t>(cuda_stream);
+    return launch_attention_backward(a);
+}
+
 rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* device_status, void* cuda_stream) {
     if (device_status == nullptr) return RPX_ERR_NULL;
     if (limit_cycles <= 0 || limit_cycles > 2000000000ll) return RPX_ERR_SHAPE;

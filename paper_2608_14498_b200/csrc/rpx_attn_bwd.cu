@@ -1,0 +1,557 @@
+// Backward of varlen causal GQA attention for sm_100a (gradients through the prefix/suffix boundary).
+//
+// With P_ij the softmax weights of query row (i,h) over keys j <= i (recomputed from the forward pass's LSE),
+// g = h / (H_q / H_kv), dP_ij = dO[i,h,:] . V[j,g,:], D_i = sum_c dO[i,h,c] O[i,h,c] (= sum_j P_ij dP_ij) and
+// dS_ij = P_ij (dP_ij - D_i):
+//     dV[j,g,:] = sum_{h in g} sum_{i >= j} P_ij  dO[i,h,:]
+//     dK[j,g,:] = scale * sum_{h in g} sum_{i >= j} dS_ij Q[i,h,:]
+//     dQ[i,h,:] = scale * sum_{j <= i} dS_ij K[j,g,:]
+// A key of the prompt receives terms from prompt queries and from response queries alike.  The query rows that take
+// part can be restricted per sequence ([q_begin, q_end)), and dK / dV can be added to what the buffers hold, so the
+// split schedule - the suffix pass's gradients first, the prefix pass's on top - is two calls of the same kernels.
+//
+// One kernel template serves both directions, because they are the same computation with the roles of the operands
+// exchanged.  An item keeps one OUTER pair of 128-row tiles (X1, X2) in shared memory and walks INNER pairs (Y1, Y2):
+//     T1 = X1 Y1^T,  T2 = X2 Y2^T          (two SS MMAs into TMEM, 128 x 128 fp32 each)
+//     element-wise: P = 2^(T1 * scale * log2 e - lse * log2 e), dS = P (T2 - D), masked; bf16 back into TMEM
+//     accumulate: A_a += P Y2, A_b += dS Y1  (TS MMAs: the TMEM tile is the A operand, Y straight from its
+//                                             [rows][d] tile as an MN-major B operand)
+//   kDq = false: (X1, X2, Y1, Y2) = (K_j, V_j, Q_i, dO_i): T1 = S^T, T2 = dP^T with keys as TMEM lanes, A_a = dV_j,
+//                A_b = dK_j; the inner loop runs over the query heads of the KV head and the query tiles i >= j.
+//   kDq = true : (X1, X2, Y1, Y2) = (Q_i, dO_i, K_j, V_j): T1 = S, T2 = dP with queries as lanes, A_b = dQ_i (A_a is
+//                not needed); the inner loop runs over the key tiles j <= i.
+// Because the transposed scores are computed directly (K Q^T instead of Q K^T), P^T and dS^T are born with keys as
+// TMEM lanes, which is what makes them usable as A operands for dV and dK without a trip through shared memory.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (it also copies the inner tile's lse and D vectors), warp 1 =
+// TMEM owner + tcgen05 issuer, warps 2..5 = element-wise + epilogue (thread = outer row = TMEM lane).
+// This first version keeps one T1/T2 pair in TMEM, so MMAs and element-wise work alternate.
+#include <math_constants.h>
+
+#include "rpx_internal.h"
+#include "rpx_ptx.cuh"
+
+namespace rpx {
+
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kStages = 2;   // inner (Y1, Y2) pairs in flight
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct Ctl {
+    uint64_t outer_full;          // producer -> issuer: X1, X2 are in shared memory
+    uint64_t outer_empty;         // issuer -> producer: the item's last T MMAs have finished
+    uint64_t in_full[kStages];
+    uint64_t in_empty[kStages];
+    uint64_t t_full;              // issuer -> element-wise warps: T1, T2 of a step are in TMEM
+    uint64_t e_ready;             // element-wise warps -> issuer: P / dS of the step are in TMEM
+    uint64_t acc_done;            // issuer -> element-wise warps: the item's last accumulate MMAs have finished
+    uint64_t acc_free;            // element-wise warps -> issuer: the accumulators have been read out
+    uint64_t drain;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t drain_flag;
+    uint32_t data_error;
+    float vec[kStages][2][kTile]; // kDq = false: (lse * log2 e, D) of the inner query tile, per stage
+};
+
+template <int D>
+struct Layout {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kHalfBytes = kTile * 128;
+    static constexpr int kTileBytes = kHalves * kHalfBytes;
+    static constexpr int kOuterOff = 0;                                  // X1, X2
+    static constexpr int kInnerOff = 2 * kTileBytes;                     // kStages x (Y1, Y2)
+    static constexpr int kCtlOff = kInnerOff + kStages * 2 * kTileBytes;
+    static constexpr size_t kSmemBytes = kCtlOff + sizeof(Ctl);
+};
+
+struct Params {
+    const int32_t* cu_seqlens;
+    const int32_t* q_begin;   // nullable: first query row of every sequence that takes part
+    const int32_t* q_end;     // nullable: one past the last
+    int32_t batch, num_q_heads, num_kv_heads, group;
+    int32_t n_tiles;          // 128-row tiles per sequence the work list covers
+    int32_t n_items;
+    int64_t total_tokens;
+    const float* lse;         // [tokens][H_q], natural log
+    const float* dvec;        // [tokens][H_q]: D = rowsum(dO * O)
+    float scale, scale_log2;
+    float* dq;                // [tokens][H_q][D]
+    float* dk;                // [tokens][H_kv][D]
+    float* dv;
+    int32_t accumulate;       // add dK / dV to what the buffers hold
+    int32_t* status;
+};
+
+struct Item {
+    int32_t seq, head, tile, tok0, len, qb, qe;
+    int32_t in_lo, in_hi, n_heads;  // inner tiles in_lo .. in_hi (inclusive) for each of n_heads heads
+    bool active, bad;
+};
+
+template <bool kDq>
+__device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
+    Item it;
+    const int32_t heads = kDq ? p.num_q_heads : p.num_kv_heads;
+    const int32_t per_tile = p.batch * heads;
+    // dkdv: early key tiles have the most query tiles behind them, dq: late query tiles the most keys: longest first
+    const int32_t t = idx / per_tile;
+    it.tile = kDq ? p.n_tiles - 1 - t : t;
+    const int32_t rem = idx % per_tile;
+    it.seq = rem / heads;
+    it.head = rem % heads;
+    it.tok0 = __ldg(p.cu_seqlens + it.seq);
+    it.len = __ldg(p.cu_seqlens + it.seq + 1) - it.tok0;
+    bool bad = it.tok0 < 0 || it.len < 0 || static_cast<int64_t>(it.tok0) + it.len > p.total_tokens;
+    it.qb = p.q_begin != nullptr ? __ldg(p.q_begin + it.seq) : 0;
+    it.qe = p.q_end != nullptr ? __ldg(p.q_end + it.seq) : it.len;
+    it.bad = bad;
+    if (bad) it.len = 0;
+    it.qb = max(0, it.qb);
+    it.qe = min(it.len, it.qe);
+    it.active = !bad && it.tile * kTile < it.len && it.qb < it.qe;
+    if (kDq) {
+        // outer = query tile: it must hold rows of the range; inner = key tiles 0 .. tile
+        it.active = it.active && it.tile * kTile < it.qe && (it.tile + 1) * kTile > it.qb;
+        it.in_lo = 0;
+        it.in_hi = it.tile;
+        it.n_heads = 1;
+    } else {
+        // outer = key tile; inner = query tiles that hold rows >= the tile's first key and inside the range
+        it.in_lo = max(it.tile, it.qb / kTile);
+        it.in_hi = (it.qe - 1) / kTile;
+        it.n_heads = p.group;
+        it.active = it.active && it.in_lo <= it.in_hi;
+    }
+    if (!it.active) it.n_heads = 0;
+    return it;
+}
+
+template <int D, bool kDq>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do, const Params p) {
+    using L = Layout<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if ((smem_u32(smem) & 1023u) != 0u) {
+        if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, RPX_ERR_CUDA);
+        return;
+    }
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + L::kCtlOff);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&ctl->outer_full, 1);
+        mbar_init(&ctl->outer_empty, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ctl->in_full[s], 1);
+            mbar_init(&ctl->in_empty[s], 1);
+        }
+        mbar_init(&ctl->t_full, 1);
+        mbar_init(&ctl->e_ready, 4);
+        mbar_init(&ctl->acc_done, 1);
+        mbar_init(&ctl->acc_free, 4);
+        mbar_init(&ctl->drain, 1);
+        ctl->abort_flag = 0;
+        ctl->drain_flag = 0;
+        ctl->data_error = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&ctl->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+    // TMEM columns: T1 at 0, T2 at 128, accumulator a at 256, accumulator b at 256 + D
+    const CUtensorMap* map_x1 = kDq ? &tmap_q : &tmap_k;
+    const CUtensorMap* map_x2 = kDq ? &tmap_do : &tmap_v;
+    const CUtensorMap* map_y1 = kDq ? &tmap_k : &tmap_q;
+    const CUtensorMap* map_y2 = kDq ? &tmap_v : &tmap_do;
+
+    if (warp == 0) {
+        // =========================================================== producer warp
+        bool ok = true;
+        uint32_t n_items = 0, n_in = 0;
+        for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+            const Item it = decode_item<kDq>(p, idx);
+            if (it.bad) ctl->data_error = 1u;  // offsets that leave the packed tensors: reported, not followed
+            if (!it.active) continue;
+            const int32_t kv_head = kDq ? it.head / p.group : it.head;
+            if (n_items > 0 && !mbar_wait(&ctl->outer_empty, (n_items - 1) & 1u, abort_flag)) {
+                ok = false;
+                break;
+            }
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&ctl->outer_full, 2 * L::kTileBytes);
+                for (int hf = 0; hf < L::kHalves; ++hf) {
+                    // x1/x2 head coordinate: K, V by KV head; Q, dO by query head
+                    tma_load_3d(smem + L::kOuterOff + hf * L::kHalfBytes, map_x1, &ctl->outer_full, hf * 64,
+                                kDq ? it.head : kv_head, it.tok0 + it.tile * kTile);
+                    tma_load_3d(smem + L::kOuterOff + L::kTileBytes + hf * L::kHalfBytes, map_x2, &ctl->outer_full, hf * 64,
+                                kDq ? it.head : kv_head, it.tok0 + it.tile * kTile);
+                }
+            }
+            for (int32_t hh = 0; ok && hh < it.n_heads; ++hh) {
+                const int32_t qh = kDq ? it.head : it.head * p.group + hh;  // the query head of this inner run
+                for (int32_t in = it.in_lo; ok && in <= it.in_hi; ++in, ++n_in) {
+                    const uint32_t stage = n_in % kStages, phase = (n_in / kStages) & 1u;
+                    if (!mbar_wait(&ctl->in_empty[stage], phase ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* y1 = smem + L::kInnerOff + stage * 2 * L::kTileBytes;
+                    uint8_t* y2 = y1 + L::kTileBytes;
+                    if (!kDq) {
+                        // lse (in log2 units) and D of the inner query tile, for the element-wise warps
+                        for (int32_t r = lane; r < kTile; r += 32) {
+                            const int32_t qr = in * kTile + r;
+                            float l2 = 0.f, dd = 0.f;
+                            if (qr < it.len) {
+                                const int64_t rh = static_cast<int64_t>(it.tok0 + qr) * p.num_q_heads + qh;
+                                l2 = __ldg(p.lse + rh) * kLog2e;
+                                dd = __ldg(p.dvec + rh);
+                            }
+                            ctl->vec[stage][0][r] = l2;
+                            ctl->vec[stage][1][r] = dd;
+                        }
+                        __syncwarp();
+                    }
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(&ctl->in_full[stage], 2 * L::kTileBytes);
+                        for (int hf = 0; hf < L::kHalves; ++hf) {
+                            tma_load_3d(y1 + hf * L::kHalfBytes, map_y1, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
+                                        it.tok0 + in * kTile);
+                            tma_load_3d(y2 + hf * L::kHalfBytes, map_y2, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
+                                        it.tok0 + in * kTile);
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+            ++n_items;
+        }
+        if (!ok) {
+            const uint32_t first = n_in > kStages ? n_in - kStages : 0u;
+            for (uint32_t i = first; i < n_in; ++i)
+                mbar_wait(&ctl->in_full[i % kStages], (i / kStages) & 1u, &ctl->drain_flag, kDrainLimitCycles);
+            if (n_items > 0) mbar_wait(&ctl->outer_full, (n_items - 1) & 1u, &ctl->drain_flag, kDrainLimitCycles);
+        }
+    } else if (warp == 1) {
+        // =========================================================== tcgen05 issuer (one thread)
+        if (elect_one()) {
+            constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kTile, false, false);
+            constexpr uint32_t idesc_acc = make_idesc_bf16(kTile, D, false, true);
+            const uint32_t outer_addr = smem_u32(smem + L::kOuterOff);
+            const uint32_t inner_addr = smem_u32(smem + L::kInnerOff);
+            const uint64_t x1_desc = make_smem_desc_sw128(outer_addr, 16, 1024);
+            const uint64_t x2_desc = make_smem_desc_sw128(outer_addr + L::kTileBytes, 16, 1024);
+            bool ok = true;
+            uint32_t n_items = 0, n_in = 0;
+            for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+                const Item it = decode_item<kDq>(p, idx);
+                if (!it.active) continue;
+                ok = mbar_wait(&ctl->outer_full, n_items & 1u, abort_flag);
+                // the accumulators still hold the previous item's result until its epilogue has read them
+                if (ok && n_items > 0) ok = mbar_wait(&ctl->acc_free, (n_items - 1) & 1u, abort_flag);
+                const int32_t steps = it.n_heads * (it.in_hi - it.in_lo + 1);
+                for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
+                    const uint32_t stage = n_in % kStages, phase = (n_in / kStages) & 1u;
+                    if (!mbar_wait(&ctl->in_full[stage], phase, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t y1_addr = inner_addr + stage * 2 * L::kTileBytes;
+                    const uint64_t y1_k = make_smem_desc_sw128(y1_addr, 16, 1024);                              // K-major
+                    const uint64_t y2_k = make_smem_desc_sw128(y1_addr + L::kTileBytes, 16, 1024);
+                    const uint64_t y1_mn = make_smem_desc_sw128(y1_addr, L::kHalfBytes, 1024);                  // MN-major
+                    const uint64_t y2_mn = make_smem_desc_sw128(y1_addr + L::kTileBytes, L::kHalfBytes, 1024);
+                    // T1 = X1 Y1^T, T2 = X2 Y2^T (in order behind the previous step's accumulate MMAs, which read P / dS
+                    // from the same columns)
+                    if (D == 128) {
+                        umma_ss_k128_overwrite(tmem_base, x1_desc, y1_k, idesc_t);
+                        umma_ss_k128_overwrite(tmem_base + kTile, x2_desc, y2_k, idesc_t);
+                    } else {
+                        umma_ss_k64_overwrite(tmem_base, x1_desc, y1_k, idesc_t);
+                        umma_ss_k64_overwrite(tmem_base + kTile, x2_desc, y2_k, idesc_t);
+                    }
+                    umma_commit(&ctl->t_full);
+                    if (s == steps - 1) umma_commit(&ctl->outer_empty);
+                    if (!mbar_wait(&ctl->e_ready, n_in & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    // accumulate: a += P Y2 (dV; not for dQ), b += dS Y1 (dK or dQ)
+                    if (!kDq) umma_ts_k128(tmem_base + 2 * kTile, tmem_base, y2_mn, idesc_acc, s != 0 ? 1u : 0u);
+                    umma_ts_k128(tmem_base + 2 * kTile + D, tmem_base + kTile, y1_mn, idesc_acc, s != 0 ? 1u : 0u);
+                    umma_commit(&ctl->in_empty[stage]);
+                    if (s == steps - 1) umma_commit(&ctl->acc_done);
+                }
+                ++n_items;
+            }
+            if (!ok) {
+                umma_commit(&ctl->drain);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, kDrainLimitCycles);
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================================================== element-wise + epilogue warps (thread = outer row)
+        const uint32_t quarter = warp & 3;
+        const int32_t r = quarter * 32 + lane;
+        const uint32_t lane_addr = (quarter * 32u) << 16;
+        const uint32_t t1 = tmem_base + lane_addr, t2 = tmem_base + kTile + lane_addr;
+        bool ok = true;
+        uint32_t n_items = 0, n_in = 0;
+        for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+            const Item it = decode_item<kDq>(p, idx);
+            if (!it.active) continue;
+            const int32_t outer_row = it.tile * kTile + r;  // key position (dK/dV) or query position (dQ)
+            float lse2_row = 0.f, d_row = 0.f;
+            bool row_ok = outer_row < it.len;
+            if (kDq) {
+                row_ok = row_ok && outer_row >= it.qb && outer_row < it.qe;
+                if (row_ok) {
+                    const int64_t rh = static_cast<int64_t>(it.tok0 + outer_row) * p.num_q_heads + it.head;
+                    lse2_row = __ldg(p.lse + rh) * kLog2e;
+                    d_row = __ldg(p.dvec + rh);
+                }
+            }
+            const int32_t n_inner = it.in_hi - it.in_lo + 1;
+            const int32_t steps = it.n_heads * n_inner;
+            for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
+                const uint32_t stage = n_in % kStages;
+                const int32_t in = it.in_lo + s % n_inner;
+                // the producer's lse / D vectors of this stage are visible once the stage's barrier has completed
+                if (!kDq && !mbar_wait(&ctl->in_full[stage], (n_in / kStages) & 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                if (!mbar_wait(&ctl->t_full, n_in & 1u, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+#pragma unroll 1
+                for (int c = 0; c < kTile / 32; ++c) {
+                    uint32_t a[32], b[32];
+                    tmem_ld32(t1 + c * 32, a);
+                    tmem_ld32(t2 + c * 32, b);
+                    tmem_ld_wait();
+                    uint32_t pw[16], dw[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float pv[2], ds[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int32_t inner_pos = in * kTile + c * 32 + i + e;  // query position (dK/dV) or key position (dQ)
+                            bool valid;
+                            float l2, dd;
+                            if (kDq) {
+                                valid = row_ok && inner_pos <= outer_row;
+                                l2 = lse2_row;
+                                dd = d_row;
+                            } else {
+                                valid = row_ok && inner_pos >= outer_row && inner_pos >= it.qb && inner_pos < it.qe;
+                                l2 = ctl->vec[stage][0][c * 32 + i + e];
+                                dd = ctl->vec[stage][1][c * 32 + i + e];
+                            }
+                            const float pe = valid ? fast_exp2(fmaf(__uint_as_float(a[i + e]), p.scale_log2, -l2)) : 0.f;
+                            pv[e] = pe;
+                            ds[e] = valid ? pe * (__uint_as_float(b[i + e]) - dd) : 0.f;
+                        }
+                        pw[i >> 1] = pack_bf16x2(pv[0], pv[1]);
+                        dw[i >> 1] = pack_bf16x2(ds[0], ds[1]);
+                    }
+                    // P over the first 64 columns of T1, dS over the first 64 of T2 (columns this thread has read)
+                    if (!kDq) tmem_st16(t1 + c * 16, pw);
+                    tmem_st16(t2 + c * 16, dw);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->e_ready);
+            }
+            if (!ok) break;
+            // ---- epilogue: the accumulators -> global (fp32), dK and dQ times the softmax scale
+            ok = mbar_wait(&ctl->acc_done, n_items & 1u, abort_flag);
+            ++n_items;
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool store = kDq ? row_ok : outer_row < it.len;
+            const int32_t out_head = it.head;
+            const int32_t out_heads = kDq ? p.num_q_heads : p.num_kv_heads;
+            const int64_t out_off = (static_cast<int64_t>(it.tok0 + outer_row) * out_heads + out_head) * D;
+#pragma unroll 1
+            for (int which = kDq ? 1 : 0; which < 2; ++which) {
+                float* dst = (which == 0 ? p.dv : (kDq ? p.dq : p.dk)) + out_off;
+                const float mul = which == 0 ? 1.f : p.scale;
+                const bool add = !kDq && p.accumulate != 0;
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t a[32];
+                    tmem_ld32(tmem_base + 2 * kTile + which * D + c * 32 + lane_addr, a);
+                    tmem_ld_wait();
+                    if (store) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            float4 v = make_float4(__uint_as_float(a[i]) * mul, __uint_as_float(a[i + 1]) * mul,
+                                                   __uint_as_float(a[i + 2]) * mul, __uint_as_float(a[i + 3]) * mul);
+                            float4* q4 = reinterpret_cast<float4*>(dst + c * 32 + i);
+                            if (add) {
+                                const float4 old = *q4;
+                                v.x += old.x;
+                                v.y += old.y;
+                                v.z += old.z;
+                                v.w += old.w;
+                            }
+                            *q4 = v;
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->acc_free);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && p.status != nullptr) {
+        if (ctl->abort_flag != 0u) atomicCAS(p.status, 0, RPX_ERR_TIMEOUT);
+        else if (ctl->data_error != 0u) atomicCAS(p.status, 0, RPX_ERR_DEVICE_DATA);
+    }
+}
+
+// D[token, head] = sum_c dO[token, head, c] * O[token, head, c]; one warp per (token, head)
+__global__ void attn_bwd_dvec_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
+                                     int64_t rows, int32_t head_dim, float* __restrict__ dvec) {
+    const int64_t row = (blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    float acc = 0.f;
+    for (int c = lane * 2; c < head_dim; c += 64) {
+        const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(out + row * head_dim + c);
+        const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(dout + row * head_dim + c);
+        acc = fmaf(__bfloat162float(o.x), __bfloat162float(g.x), acc);
+        acc = fmaf(__bfloat162float(o.y), __bfloat162float(g.y), acc);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (lane == 0) dvec[row] = acc;
+}
+
+// rows of dK / dV no key tile's item writes (sequences outside every range): cleared when not accumulating
+__global__ void attn_bwd_zero_kernel(float* __restrict__ a, float* __restrict__ b, int64_t n) {
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        a[i] = 0.f;
+        if (b != nullptr) b[i] = 0.f;
+    }
+}
+
+template <int D>
+rpx_status_t launch_d(const AttnBwdArgs& a) {
+    using L = Layout<D>;
+    CUtensorMap tq, tk, tv, tdo;
+    const uint64_t tokens = static_cast<uint64_t>(a.total_tokens);
+    const uint32_t box[3] = {64, 1, kTile};
+    {
+        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_q_heads), tokens};
+        const uint64_t qs[2] = {D * 2ull, static_cast<uint64_t>(a.q_tok_stride) * 2};
+        const uint64_t os[2] = {D * 2ull, static_cast<uint64_t>(a.num_q_heads) * D * 2ull};
+        if (rpx_status_t rc = encode_tmap_bf16(&tq, a.q, 3, dims, qs, box)) return rc;
+        if (rpx_status_t rc = encode_tmap_bf16(&tdo, a.dout, 3, dims, os, box)) return rc;
+    }
+    {
+        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_kv_heads), tokens};
+        const uint64_t ks[2] = {D * 2ull, static_cast<uint64_t>(a.k_tok_stride) * 2};
+        const uint64_t vs[2] = {D * 2ull, static_cast<uint64_t>(a.v_tok_stride) * 2};
+        if (rpx_status_t rc = encode_tmap_bf16(&tk, a.k, 3, dims, ks, box)) return rc;
+        if (rpx_status_t rc = encode_tmap_bf16(&tv, a.v, 3, dims, vs, box)) return rc;
+    }
+    int sms = sm_count();
+    if (sms <= 0) return RPX_ERR_CUDA;
+    if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;
+    // ---- D = rowsum(dO * O)
+    const int64_t rows = a.total_tokens * a.num_q_heads;
+    {
+        const int threads = 256;
+        const int64_t blocks = (rows * 32 + threads - 1) / threads;
+        attn_bwd_dvec_kernel<<<static_cast<unsigned>(blocks), threads, 0, a.stream>>>(
+            static_cast<const __nv_bfloat16*>(a.out), static_cast<const __nv_bfloat16*>(a.dout), rows, D, a.dvec);
+        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    }
+    const int64_t n_q = a.total_tokens * a.num_q_heads * D, n_kv = a.total_tokens * a.num_kv_heads * D;
+    attn_bwd_zero_kernel<<<sms * 4, 256, 0, a.stream>>>(a.dq, nullptr, n_q);
+    if (!a.accumulate) attn_bwd_zero_kernel<<<sms * 4, 256, 0, a.stream>>>(a.dk, a.dv, n_kv);
+    if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+
+    Params p;
+    p.cu_seqlens = a.cu_seqlens;
+    p.q_begin = a.q_begin;
+    p.q_end = a.q_end;
+    p.batch = a.batch;
+    p.num_q_heads = a.num_q_heads;
+    p.num_kv_heads = a.num_kv_heads;
+    p.group = a.num_q_heads / a.num_kv_heads;
+    p.n_tiles = (a.max_seqlen + kTile - 1) / kTile;
+    p.total_tokens = a.total_tokens;
+    p.lse = a.lse;
+    p.dvec = a.dvec;
+    p.scale = a.softmax_scale > 0.f ? a.softmax_scale : 1.0f / sqrtf(static_cast<float>(D));
+    p.scale_log2 = p.scale * kLog2e;
+    p.dq = a.dq;
+    p.dk = a.dk;
+    p.dv = a.dv;
+    p.accumulate = a.accumulate ? 1 : 0;
+    p.status = a.device_status;
+    if (cudaFuncSetAttribute(attn_bwd_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(L::kSmemBytes)) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_bwd_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(L::kSmemBytes)) != cudaSuccess)
+        return RPX_ERR_CUDA;
+    {
+        const int64_t items = static_cast<int64_t>(p.n_tiles) * a.batch * a.num_kv_heads;
+        if (items > INT32_MAX) return RPX_ERR_SHAPE;
+        p.n_items = static_cast<int32_t>(items);
+        const unsigned grid = static_cast<unsigned>(items < sms ? items : sms);
+        attn_bwd_kernel<D, false><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tdo, p);
+        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    }
+    {
+        const int64_t items = static_cast<int64_t>(p.n_tiles) * a.batch * a.num_q_heads;
+        if (items > INT32_MAX) return RPX_ERR_SHAPE;
+        p.n_items = static_cast<int32_t>(items);
+        const unsigned grid = static_cast<unsigned>(items < sms ? items : sms);
+        attn_bwd_kernel<D, true><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tdo, p);
+        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    }
+    return RPX_OK;
+}
+
+}  // namespace
+
+rpx_status_t launch_attention_backward(const AttnBwdArgs& a) {
+    if (a.total_tokens == 0 || a.batch == 0 || a.max_seqlen == 0) return RPX_OK;
+    if (a.head_dim == 128) return launch_d<128>(a);
+    if (a.head_dim == 64) return launch_d<64>(a);
+    return RPX_ERR_SHAPE;
+}
+
+}  // namespace rpx

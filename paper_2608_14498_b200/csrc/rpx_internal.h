@@ -93,6 +93,26 @@ int64_t logprob_backward_block_rows(int64_t n_tokens);
 size_t logprob_backward_workspace(int64_t n_tokens, int32_t vocab);
 rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a);
 
+struct AttnBwdArgs {
+    int32_t num_q_heads, num_kv_heads, head_dim;
+    float softmax_scale;
+    const void *q, *k, *v;      // bf16, packed whole sequences
+    int64_t q_tok_stride, k_tok_stride, v_tok_stride;
+    const void *out, *dout;     // bf16 [tokens][H_q][d], contiguous
+    const float* lse;           // [tokens][H_q]
+    const int32_t* cu_seqlens;
+    const int32_t *q_begin, *q_end;  // nullable: the query rows of every sequence that take part
+    int32_t batch;
+    int64_t total_tokens;
+    int32_t max_seqlen;
+    float *dq, *dk, *dv;        // fp32
+    bool accumulate;            // add dK / dV to what the buffers hold
+    float* dvec;                // workspace: fp32 [tokens][H_q]
+    int32_t* device_status;
+    cudaStream_t stream;
+};
+rpx_status_t launch_attention_backward(const AttnBwdArgs& a);
+
 rpx_status_t launch_bounded_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t stream);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

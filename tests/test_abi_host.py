@@ -121,6 +121,30 @@ def test_attention_rejects_bad_arguments_before_any_launch(lib):
     assert rc == -1  # cached_lens missing
 
 
+def test_attention_backward_rejects_bad_arguments_before_any_launch(lib):
+    def call(desc=None, q=0x1000, dout=0x1000, lse=0x1000, dq=0x1000, strides=(512, 256, 256), total=16, ws=0x10000,
+             ws_bytes=1 << 20, batch=1):
+        desc = desc or B.AttnDesc(4, 2, 128, 0.0, B.RPX_BF16)
+        return lib.rpx_attn_backward(ctypes.byref(desc), q, 0x1000, 0x1000, strides[0], strides[1], strides[2], 0x1000,
+                                     dout, lse, 0x1000, None, None, batch, total, 16, dq, 0x1000, 0x1000, 0, ws, ws_bytes,
+                                     None, None)
+
+    assert call(desc=B.AttnDesc(4, 2, 128, 0.0, B.RPX_F32)) == -3   # bf16 only
+    assert call(desc=B.AttnDesc(4, 3, 128, 0.0, B.RPX_BF16)) == -2
+    assert call(q=None) == -1
+    assert call(dout=None) == -1
+    assert call(lse=None) == -1
+    assert call(dq=0x1008) == -4
+    assert call(strides=(256, 256, 256)) == -2
+    assert call(ws=None) == -5
+    assert call(ws_bytes=16) == -5          # 16 tokens x 4 heads x 4 bytes = 256 are needed
+    assert call(ws=0x10010) == -4
+    assert call(total=0, q=None) == 0 and call(batch=0, q=None) == 0
+    good = B.AttnDesc(28, 4, 128, 0.0, B.RPX_BF16)
+    assert lib.rpx_attn_backward_workspace_bytes(ctypes.byref(good), 1000) == 112128  # 1000 x 28 x 4 = 112000 rounded up to 256
+    assert lib.rpx_attn_backward_workspace_bytes(ctypes.byref(good), 3) == 512
+
+
 def test_logprobs_rejects_bad_arguments_before_any_launch(lib):
     def call(hidden=0x1000, stride=256, w=0x1000, ids=0x1000, n=8, h=256, v=4096, dt=B.RPX_BF16, lp=0x1000, ws=0x1000,
              ws_bytes=1 << 30):
