@@ -2,7 +2,7 @@
 """Benchmark of the prefix+suffix scoring hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3]
-    python bench.py --profile-case lm|lmbwd|prefix|suffix [--reps 3]      (small launches for profiler captures)
+    python bench.py --profile-case lm|lmbwd|prefix|suffix|attnbwd [--reps 3]      (small launches for profiler captures)
 
 One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
 boundary-KV write), prefix log-probs, suffix attention over the cached KV, suffix log-probs.
@@ -407,6 +407,69 @@ def measure_backward(torch, config, local_rank, reps=3):
             "gpu_launches": 2 * reps * -(-n // 9472), "clocks": clocks}
 
 
+def measure_attn_backward(torch, config, local_rank, reps=60):
+    """rpx_attn_backward over the whole sequences (prompt then response) of one config, with out and lse from the
+    library's forward pass: milliseconds; TFLOP/s on the algorithmic flops (five products per causal tile pair: S, dP,
+    dV, dK, dQ = 2.5 x the forward pass) and on the executed ones (seven: the dQ kernel recomputes S and dP)."""
+    import paper_2608_14498_b200 as rpx
+    from paper_2608_14498_b200 import binding as B
+
+    dev = torch.device("cuda", local_rank)
+    cfg = wk.CONFIGS[config]
+    wl = wk.make_workload(cfg, seed=0, lm=False)
+
+    def t(a):
+        x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return x.to(dev)
+
+    q, k, v, cu = t(wl.q), t(wl.k), t(wl.v), t(wl.cu_full)
+    dout = t(wk.make_workload(cfg, seed=1, lm=False).q)  # an upstream gradient with the same distribution as q
+    lens = (wl.prompt_lens + wl.response_lens).astype(np.int64)
+    max_len, n = int(lens.max()), int(lens.sum())
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out, lse = rpx.prefix_attn(q, k, v, cu, max_len, return_lse=True, device_status=status)
+    dq = torch.empty(tuple(q.shape), dtype=torch.float32, device=dev)
+    dk = torch.empty(tuple(k.shape), dtype=torch.float32, device=dev)
+    dvv = torch.empty_like(dk)
+    ws = torch.empty(B.attn_backward_workspace_bytes(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, n), dtype=torch.uint8,
+                     device=dev)
+
+    def call():
+        rpx.attn_backward(q, k, v, out, dout, lse, cu, max_len, dq=dq, dk=dk, dv=dvv, workspace=ws, device_status=status)
+
+    for _ in range(2):
+        call()
+    torch.cuda.synchronize()
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(local_rank).uuid)
+        gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark()
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.mark()
+    clocks = sampler.stop()
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} in the attention backward pass")
+    ms = e0.elapsed_time(e1) / reps
+    peaks = load_peaks()
+    fwd = float((4.0 * cfg.head_dim * cfg.num_q_heads * (lens * (lens + 1) / 2)).sum())
+    tf, tf_exec = 2.5 * fwd / (ms * 1e-3) / 1e12, 3.5 * fwd / (ms * 1e-3) / 1e12
+    sustained = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    return {"what": "rpx_attn_backward over the whole sequences (D, clears, the dK/dV kernel, the dQ kernel)",
+            "workload": cfg.name, "tokens": n, "ms": ms, "tflops": tf, "tflops_executed": tf_exec,
+            "frac_of_sustained_peak": tf / sustained, "executed_frac_of_sustained_peak": tf_exec / sustained,
+            "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]), "workspace_bytes": ws.numel(),
+            "gpu_launches": 5 * reps, "clocks": clocks}
+
+
 def run_ours(args, rank, local_rank, world):
     import torch
     import torch.distributed as dist
@@ -438,7 +501,9 @@ def run_ours(args, rank, local_rank, world):
     backward = None
     if world == 1 and not args.no_backward:
         torch.cuda.empty_cache()
-        backward = measure_backward(torch, "C2", local_rank)
+        backward = {"lm_head": measure_backward(torch, "C2", local_rank)}
+        torch.cuda.empty_cache()
+        backward["attention"] = measure_attn_backward(torch, "C2", local_rank)
     if rank == 0:
         line = {
             "metric": "scored_tokens_per_s", "value": head["value"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -463,7 +528,9 @@ def run_profile_case(args):
       lm      8192 rows x 32768 vocabulary columns, hidden 3584  (7B-shaped slice of the LM head)
       lmbwd   the same slice through rpx_token_logprobs_backward (two kernels per launch: dL/dz, then dhidden)
       prefix  4 sequences x 4096 prompt tokens, 28 query / 4 KV heads, head_dim 128, with cache write
-      suffix  the same 4 prompts cached, 256 response tokens each"""
+      suffix  the same 4 prompts cached, 256 response tokens each
+      attnbwd rpx_attn_backward over the same 4 sequences whole (4352 tokens each): D, two clears, the dK/dV kernel,
+              the dQ kernel per launch"""
     import torch
 
     import paper_2608_14498_b200 as rpx
@@ -491,6 +558,14 @@ def run_profile_case(args):
         g = torch.ones(h.shape[0], dtype=torch.float32, device=dev)
         for _ in range(1 + args.reps):
             rpx.token_logprobs_backward(h, w, ids, lse, g, device_status=status)
+    elif case == "attnbwd":
+        cfg = wk.Config("profile-attn", "bf16", 4, 28, 4, 128, 3584, 1024, ("fixed", 4096), ("fixed", 256))
+        wl = wk.make_workload(cfg, seed=0, lm=False)
+        q, k, v, cu = dv(wl.q), dv(wl.k), dv(wl.v), dv(wl.cu_full)
+        out, lse = rpx.prefix_attn(q, k, v, cu, 4352, return_lse=True, device_status=status)
+        dout = dv(wk.make_workload(cfg, seed=1, lm=False).q)
+        for _ in range(1 + args.reps):
+            rpx.attn_backward(q, k, v, out, dout, lse, cu, 4352, device_status=status)
     else:
         cfg = wk.Config("profile-attn", "bf16", 4, 28, 4, 128, 3584, 1024, ("fixed", 4096), ("fixed", 256))
         wl = wk.make_workload(cfg, seed=0, lm=False)
@@ -593,7 +668,7 @@ def main():
     ap.add_argument("--config", default="C3", choices=sorted(wk.CONFIGS), help="headline workload (C3 = the largest single-GPU config)")
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
     ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
-    ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix", "attnbwd"], help="launch one kernel a few times on a small case and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")

@@ -6,6 +6,8 @@ or eager fallback: a missing library or a non-sm_100 device is an error.
 """
 from .binding import (  # noqa: F401
     RpxError,
+    attn_backward,
+    attn_backward_workspace_bytes,
     chunk_attn,
     get_sm_budget,
     library_path,
@@ -18,7 +20,6 @@ from .binding import (  # noqa: F401
     suffix_attn,
     suffix_attn_workspace_bytes,
     token_logprobs,
-    attn_backward,
     token_logprobs_backward,
     token_logprobs_backward_workspace_bytes,
     token_logprobs_merge,

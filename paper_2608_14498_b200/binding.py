@@ -230,6 +230,11 @@ def suffix_attn_workspace_bytes(num_q_heads, num_kv_heads, head_dim, dtype_code,
     return int(load_library().rpx_suffix_attn_workspace_bytes(ctypes.byref(d), int(total_tokens)))
 
 
+def attn_backward_workspace_bytes(num_q_heads, num_kv_heads, head_dim, total_tokens) -> int:
+    desc = AttnDesc(num_q_heads, num_kv_heads, head_dim, 0.0, RPX_BF16)
+    return int(load_library().rpx_attn_backward_workspace_bytes(ctypes.byref(desc), int(total_tokens)))
+
+
 def token_logprobs_workspace_bytes(n_tokens, hidden_dim, vocab, dtype_code) -> int:
     return int(load_library().rpx_token_logprobs_workspace_bytes(int(n_tokens), int(hidden_dim), int(vocab),
                                                                  int(dtype_code)))

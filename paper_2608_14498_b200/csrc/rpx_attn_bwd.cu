@@ -23,9 +23,15 @@
 // Because the transposed scores are computed directly (K Q^T instead of Q K^T), P^T and dS^T are born with keys as
 // TMEM lanes, which is what makes them usable as A operands for dV and dK without a trip through shared memory.
 //
-// Warp roles (192 threads): warp 0 = TMA producer (it also copies the inner tile's lse and D vectors), warp 1 =
-// TMEM owner + tcgen05 issuer, warps 2..5 = element-wise + epilogue (thread = outer row = TMEM lane).
-// This first version keeps one T1/T2 pair in TMEM, so MMAs and element-wise work alternate.
+// Warp roles (320 threads): warp 0 = TMA producer (it also copies the inner tile's lse and D vectors), warp 1 =
+// TMEM owner + tcgen05 issuer, warps 2..9 = element-wise + epilogue (thread = outer row = TMEM lane; two warps per
+// lane quarter, each taking half of the columns).
+// TMEM holds the two accumulators (2 x d columns) and ONE T1/T2 pair (256 columns), so to overlap tensor-core and
+// element-wise work an inner tile is processed as two halves of 64 inner rows: while the warps turn half a into
+// P / dS, the tensor core computes T of half b, then accumulates half a, then computes the next step's half a, ...
+// Masking costs nothing off the diagonal: rows of the inner query tile that do not take part get -lse = -inf (P = 0,
+// dS = 0) in the vector the producer prepares, and outer rows that do not exist only pollute their own accumulator
+// lanes, which are never stored; only the diagonal tile applies the causal predicate per element.
 #include <math_constants.h>
 
 #include "rpx_internal.h"
@@ -37,7 +43,8 @@ namespace {
 
 constexpr int kTile = 128;
 constexpr int kStages = 2;   // inner (Y1, Y2) pairs in flight
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kHalf = 64;    // inner rows per half step
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -46,8 +53,8 @@ struct Ctl {
     uint64_t outer_empty;         // issuer -> producer: the item's last T MMAs have finished
     uint64_t in_full[kStages];
     uint64_t in_empty[kStages];
-    uint64_t t_full;              // issuer -> element-wise warps: T1, T2 of a step are in TMEM
-    uint64_t e_ready;             // element-wise warps -> issuer: P / dS of the step are in TMEM
+    uint64_t t_full[2];           // issuer -> element-wise warps: T1, T2 of a half step are in TMEM
+    uint64_t e_ready[2];          // element-wise warps -> issuer: P / dS of the half step are in TMEM
     uint64_t acc_done;            // issuer -> element-wise warps: the item's last accumulate MMAs have finished
     uint64_t acc_free;            // element-wise warps -> issuer: the accumulators have been read out
     uint64_t drain;
@@ -55,7 +62,7 @@ struct Ctl {
     uint32_t abort_flag;
     uint32_t drain_flag;
     uint32_t data_error;
-    float vec[kStages][2][kTile]; // kDq = false: (lse * log2 e, D) of the inner query tile, per stage
+    float vec[kStages][2][kTile]; // kDq = false: (-lse * log2 e or -inf, -D) of the inner query tile, per stage
 };
 
 template <int D>
@@ -92,6 +99,31 @@ struct Item {
     int32_t in_lo, in_hi, n_heads;  // inner tiles in_lo .. in_hi (inclusive) for each of n_heads heads
     bool active, bad;
 };
+
+// Four K=16 steps of D (+)= A[tmem] * B[smem, MN-major] over 64 inner rows.  The A operand of steps 0, 1 sits in
+// columns 0..15 and that of steps 2, 3 in columns 32..47 (each warp group leaves its 16 packed columns at the start of
+// the 32 it has read); B advances 16 rows of 128 bytes (128 units) per step.
+__device__ __forceinline__ void umma_ts_k64_split(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                                  uint32_t accumulate_first) {
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 db;\n"
+        ".reg .b32 ta;\n"
+        "setp.ne.b32 pf, %4, 0;\n"
+        "setp.eq.b32 pt, %4, %4;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, pf;\n" RPX_UMMA_TS_STEP(8, 128) RPX_UMMA_TS_STEP(32, 256)
+            RPX_UMMA_TS_STEP(40, 384) "}\n" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+
+// Items are ordered longest first; the CTAs take them in serpentine order (0 .. G-1, then G-1 .. 0, ...), which
+// evens out the inner steps per CTA far better than a plain stride when the item lengths fall linearly.
+__device__ __forceinline__ int32_t item_of_round(int32_t rnd) {
+    const int32_t g = static_cast<int32_t>(gridDim.x), b = static_cast<int32_t>(blockIdx.x);
+    return rnd * g + ((rnd & 1) ? g - 1 - b : b);
+}
 
 template <bool kDq>
 __device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
@@ -153,10 +185,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_init(&ctl->in_full[s], 1);
             mbar_init(&ctl->in_empty[s], 1);
         }
-        mbar_init(&ctl->t_full, 1);
-        mbar_init(&ctl->e_ready, 4);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&ctl->t_full[h], 1);
+            mbar_init(&ctl->e_ready[h], 8);
+        }
         mbar_init(&ctl->acc_done, 1);
-        mbar_init(&ctl->acc_free, 4);
+        mbar_init(&ctl->acc_free, 8);
         mbar_init(&ctl->drain, 1);
         ctl->abort_flag = 0;
         ctl->drain_flag = 0;
@@ -181,7 +215,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // =========================================================== producer warp
         bool ok = true;
         uint32_t n_items = 0, n_in = 0;
-        for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+        for (int32_t rnd = 0, idx = blockIdx.x; ok && idx < p.n_items; idx = item_of_round(++rnd)) {
             const Item it = decode_item<kDq>(p, idx);
             if (it.bad) ctl->data_error = 1u;  // offsets that leave the packed tensors: reported, not followed
             if (!it.active) continue;
@@ -211,14 +245,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     uint8_t* y1 = smem + L::kInnerOff + stage * 2 * L::kTileBytes;
                     uint8_t* y2 = y1 + L::kTileBytes;
                     if (!kDq) {
-                        // lse (in log2 units) and D of the inner query tile, for the element-wise warps
+                        // -lse (in log2 units) and -D of the inner query tile, for the element-wise warps
                         for (int32_t r = lane; r < kTile; r += 32) {
                             const int32_t qr = in * kTile + r;
-                            float l2 = 0.f, dd = 0.f;
-                            if (qr < it.len) {
+                            float l2 = -CUDART_INF_F, dd = 0.f;  // a row that takes no part: P = 2^(-inf) = 0, dS = 0
+                            if (qr >= it.qb && qr < it.qe) {
                                 const int64_t rh = static_cast<int64_t>(it.tok0 + qr) * p.num_q_heads + qh;
-                                l2 = __ldg(p.lse + rh) * kLog2e;
-                                dd = __ldg(p.dvec + rh);
+                                l2 = -__ldg(p.lse + rh) * kLog2e;
+                                dd = -__ldg(p.dvec + rh);
                             }
                             ctl->vec[stage][0][r] = l2;
                             ctl->vec[stage][1][r] = dd;
@@ -248,55 +282,76 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     } else if (warp == 1) {
         // =========================================================== tcgen05 issuer (one thread)
         if (elect_one()) {
-            constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kTile, false, false);
+            constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kHalf, false, false);
             constexpr uint32_t idesc_acc = make_idesc_bf16(kTile, D, false, true);
+            constexpr uint32_t kHalfUnits = kHalf * 128 / 16;  // 64 rows of 128 bytes, in descriptor units of 16 bytes
             const uint32_t outer_addr = smem_u32(smem + L::kOuterOff);
             const uint32_t inner_addr = smem_u32(smem + L::kInnerOff);
             const uint64_t x1_desc = make_smem_desc_sw128(outer_addr, 16, 1024);
             const uint64_t x2_desc = make_smem_desc_sw128(outer_addr + L::kTileBytes, 16, 1024);
+            // T1 = X1 Y1^T and T2 = X2 Y2^T for the inner rows 64 h .. 64 h + 63 of the pair in `stage`
+            auto issue_t = [&](uint32_t stage, int h) {
+                const uint32_t y1_addr = inner_addr + stage * 2 * L::kTileBytes;
+                const uint64_t y1_k = make_smem_desc_sw128(y1_addr, 16, 1024) + h * kHalfUnits;
+                const uint64_t y2_k = make_smem_desc_sw128(y1_addr + L::kTileBytes, 16, 1024) + h * kHalfUnits;
+                if (D == 128) {
+                    umma_ss_k128_overwrite(tmem_base + h * kHalf, x1_desc, y1_k, idesc_t);
+                    umma_ss_k128_overwrite(tmem_base + kTile + h * kHalf, x2_desc, y2_k, idesc_t);
+                } else {
+                    umma_ss_k64_overwrite(tmem_base + h * kHalf, x1_desc, y1_k, idesc_t);
+                    umma_ss_k64_overwrite(tmem_base + kTile + h * kHalf, x2_desc, y2_k, idesc_t);
+                }
+                umma_commit(&ctl->t_full[h]);
+            };
             bool ok = true;
             uint32_t n_items = 0, n_in = 0;
-            for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+            for (int32_t rnd = 0, idx = blockIdx.x; ok && idx < p.n_items; idx = item_of_round(++rnd)) {
                 const Item it = decode_item<kDq>(p, idx);
                 if (!it.active) continue;
                 ok = mbar_wait(&ctl->outer_full, n_items & 1u, abort_flag);
                 // the accumulators still hold the previous item's result until its epilogue has read them
                 if (ok && n_items > 0) ok = mbar_wait(&ctl->acc_free, (n_items - 1) & 1u, abort_flag);
                 const int32_t steps = it.n_heads * (it.in_hi - it.in_lo + 1);
-                for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
-                    const uint32_t stage = n_in % kStages, phase = (n_in / kStages) & 1u;
-                    if (!mbar_wait(&ctl->in_full[stage], phase, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
+                if (ok) ok = mbar_wait(&ctl->in_full[n_in % kStages], (n_in / kStages) & 1u, abort_flag);
+                if (ok) {
                     tc_fence_after_sync();
+                    issue_t(n_in % kStages, 0);
+                    issue_t(n_in % kStages, 1);
+                    if (steps == 1) umma_commit(&ctl->outer_empty);
+                }
+                for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
+                    const uint32_t stage = n_in % kStages;
                     const uint32_t y1_addr = inner_addr + stage * 2 * L::kTileBytes;
-                    const uint64_t y1_k = make_smem_desc_sw128(y1_addr, 16, 1024);                              // K-major
-                    const uint64_t y2_k = make_smem_desc_sw128(y1_addr + L::kTileBytes, 16, 1024);
                     const uint64_t y1_mn = make_smem_desc_sw128(y1_addr, L::kHalfBytes, 1024);                  // MN-major
                     const uint64_t y2_mn = make_smem_desc_sw128(y1_addr + L::kTileBytes, L::kHalfBytes, 1024);
-                    // T1 = X1 Y1^T, T2 = X2 Y2^T (in order behind the previous step's accumulate MMAs, which read P / dS
-                    // from the same columns)
-                    if (D == 128) {
-                        umma_ss_k128_overwrite(tmem_base, x1_desc, y1_k, idesc_t);
-                        umma_ss_k128_overwrite(tmem_base + kTile, x2_desc, y2_k, idesc_t);
-                    } else {
-                        umma_ss_k64_overwrite(tmem_base, x1_desc, y1_k, idesc_t);
-                        umma_ss_k64_overwrite(tmem_base + kTile, x2_desc, y2_k, idesc_t);
+                    for (int h = 0; ok && h < 2; ++h) {
+                        if (!mbar_wait(&ctl->e_ready[h], n_in & 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        // accumulate over the 64 inner rows of the half: a += P Y2 (dV; not for dQ), b += dS Y1 (dK or dQ)
+                        const uint32_t acc = (s != 0 || h != 0) ? 1u : 0u;
+                        if (!kDq)
+                            umma_ts_k64_split(tmem_base + 2 * kTile, tmem_base + h * kHalf, y2_mn + h * kHalfUnits, idesc_acc, acc);
+                        umma_ts_k64_split(tmem_base + 2 * kTile + D, tmem_base + kTile + h * kHalf, y1_mn + h * kHalfUnits,
+                                          idesc_acc, acc);
+                        if (h == 1) umma_commit(&ctl->in_empty[stage]);
+                        if (s + 1 < steps) {
+                            // the next step's T of this half, in order behind the accumulate MMAs that read P / dS from
+                            // the same columns
+                            const uint32_t nstage = (n_in + 1) % kStages;
+                            if (h == 0 && !mbar_wait(&ctl->in_full[nstage], ((n_in + 1) / kStages) & 1u, abort_flag)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after_sync();
+                            issue_t(nstage, h);
+                            if (h == 1 && s + 2 == steps) umma_commit(&ctl->outer_empty);
+                        }
                     }
-                    umma_commit(&ctl->t_full);
-                    if (s == steps - 1) umma_commit(&ctl->outer_empty);
-                    if (!mbar_wait(&ctl->e_ready, n_in & 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after_sync();
-                    // accumulate: a += P Y2 (dV; not for dQ), b += dS Y1 (dK or dQ)
-                    if (!kDq) umma_ts_k128(tmem_base + 2 * kTile, tmem_base, y2_mn, idesc_acc, s != 0 ? 1u : 0u);
-                    umma_ts_k128(tmem_base + 2 * kTile + D, tmem_base + kTile, y1_mn, idesc_acc, s != 0 ? 1u : 0u);
-                    umma_commit(&ctl->in_empty[stage]);
-                    if (s == steps - 1) umma_commit(&ctl->acc_done);
                 }
+                if (ok) umma_commit(&ctl->acc_done);
                 ++n_items;
             }
             if (!ok) {
@@ -308,79 +363,86 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     } else {
         // =========================================================== element-wise + epilogue warps (thread = outer row)
         const uint32_t quarter = warp & 3;
+        const uint32_t grp = (warp - 2) >> 2;  // which 32 of a half's 64 columns
         const int32_t r = quarter * 32 + lane;
         const uint32_t lane_addr = (quarter * 32u) << 16;
         const uint32_t t1 = tmem_base + lane_addr, t2 = tmem_base + kTile + lane_addr;
+        const uint64_t sl2 = f2_pack(p.scale_log2, p.scale_log2);
         bool ok = true;
         uint32_t n_items = 0, n_in = 0;
-        for (int32_t idx = blockIdx.x; ok && idx < p.n_items; idx += gridDim.x) {
+        for (int32_t rnd = 0, idx = blockIdx.x; ok && idx < p.n_items; idx = item_of_round(++rnd)) {
             const Item it = decode_item<kDq>(p, idx);
             if (!it.active) continue;
             const int32_t outer_row = it.tile * kTile + r;  // key position (dK/dV) or query position (dQ)
-            float lse2_row = 0.f, d_row = 0.f;
-            bool row_ok = outer_row < it.len;
-            if (kDq) {
-                row_ok = row_ok && outer_row >= it.qb && outer_row < it.qe;
-                if (row_ok) {
-                    const int64_t rh = static_cast<int64_t>(it.tok0 + outer_row) * p.num_q_heads + it.head;
-                    lse2_row = __ldg(p.lse + rh) * kLog2e;
-                    d_row = __ldg(p.dvec + rh);
-                }
+            // rows of the outer tile that do not exist or take no part pollute only their own accumulator lanes, which
+            // are not stored
+            const bool row_ok = kDq ? (outer_row >= it.qb && outer_row < it.qe) : outer_row < it.len;
+            uint64_t nl2_row = 0, nd_row = 0;
+            if (kDq && row_ok) {
+                const int64_t rh = static_cast<int64_t>(it.tok0 + outer_row) * p.num_q_heads + it.head;
+                const float l2 = -__ldg(p.lse + rh) * kLog2e, nd = -__ldg(p.dvec + rh);
+                nl2_row = f2_pack(l2, l2);
+                nd_row = f2_pack(nd, nd);
             }
             const int32_t n_inner = it.in_hi - it.in_lo + 1;
             const int32_t steps = it.n_heads * n_inner;
             for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
                 const uint32_t stage = n_in % kStages;
                 const int32_t in = it.in_lo + s % n_inner;
+                const bool diagonal = in == it.tile;
                 // the producer's lse / D vectors of this stage are visible once the stage's barrier has completed
                 if (!kDq && !mbar_wait(&ctl->in_full[stage], (n_in / kStages) & 1u, abort_flag)) {
                     ok = false;
                     break;
                 }
-                if (!mbar_wait(&ctl->t_full, n_in & 1u, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after_sync();
-#pragma unroll 1
-                for (int c = 0; c < kTile / 32; ++c) {
+                for (int h = 0; h < 2; ++h) {
+                    if (!mbar_wait(&ctl->t_full[h], n_in & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t col = h * kHalf + grp * 32;  // this thread's 32 inner rows of the step
                     uint32_t a[32], b[32];
-                    tmem_ld32(t1 + c * 32, a);
-                    tmem_ld32(t2 + c * 32, b);
+                    tmem_ld32(t1 + col, a);
+                    tmem_ld32(t2 + col, b);
                     tmem_ld_wait();
                     uint32_t pw[16], dw[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        float pv[2], ds[2];
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int32_t inner_pos = in * kTile + c * 32 + i + e;  // query position (dK/dV) or key position (dQ)
-                            bool valid;
-                            float l2, dd;
-                            if (kDq) {
-                                valid = row_ok && inner_pos <= outer_row;
-                                l2 = lse2_row;
-                                dd = d_row;
-                            } else {
-                                valid = row_ok && inner_pos >= outer_row && inner_pos >= it.qb && inner_pos < it.qe;
-                                l2 = ctl->vec[stage][0][c * 32 + i + e];
-                                dd = ctl->vec[stage][1][c * 32 + i + e];
-                            }
-                            const float pe = valid ? fast_exp2(fmaf(__uint_as_float(a[i + e]), p.scale_log2, -l2)) : 0.f;
-                            pv[e] = pe;
-                            ds[e] = valid ? pe * (__uint_as_float(b[i + e]) - dd) : 0.f;
+                        uint64_t nl2, nd;
+                        if (kDq) {
+                            nl2 = nl2_row;
+                            nd = nd_row;
+                        } else {
+                            const float2 lv = *reinterpret_cast<const float2*>(&ctl->vec[stage][0][col + i]);
+                            const float2 dv2 = *reinterpret_cast<const float2*>(&ctl->vec[stage][1][col + i]);
+                            nl2 = f2_pack(lv.x, lv.y);
+                            nd = f2_pack(dv2.x, dv2.y);
                         }
-                        pw[i >> 1] = pack_bf16x2(pv[0], pv[1]);
-                        dw[i >> 1] = pack_bf16x2(ds[0], ds[1]);
+                        // P = 2^(T1 * scale * log2 e - lse * log2 e), dS = P (T2 - D), two elements per instruction
+                        float x0, x1;
+                        f2_unpack(f2_fma(f2_pack(__uint_as_float(a[i]), __uint_as_float(a[i + 1])), sl2, nl2), x0, x1);
+                        if (diagonal) {  // causal: the key position must not exceed the query position
+                            const int32_t inner_pos = in * kTile + col + i;
+                            const bool v0 = kDq ? inner_pos <= outer_row : inner_pos >= outer_row;
+                            const bool v1 = kDq ? inner_pos + 1 <= outer_row : inner_pos + 1 >= outer_row;
+                            x0 = v0 ? x0 : -CUDART_INF_F;
+                            x1 = v1 ? x1 : -CUDART_INF_F;
+                        }
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        float d0, d1;
+                        f2_unpack(f2_add(f2_pack(__uint_as_float(b[i]), __uint_as_float(b[i + 1])), nd), d0, d1);
+                        pw[i >> 1] = pack_bf16x2(p0, p1);
+                        dw[i >> 1] = pack_bf16x2(p0 * d0, p1 * d1);
                     }
-                    // P over the first 64 columns of T1, dS over the first 64 of T2 (columns this thread has read)
-                    if (!kDq) tmem_st16(t1 + c * 16, pw);
-                    tmem_st16(t2 + c * 16, dw);
+                    // P over the first 16 of the 32 columns this thread has read from T1, dS likewise in T2
+                    if (!kDq) tmem_st16(t1 + col, pw);
+                    tmem_st16(t2 + col, dw);
+                    tmem_st_wait();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->e_ready[h]);
                 }
-                tmem_st_wait();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->e_ready);
             }
             if (!ok) break;
             // ---- epilogue: the accumulators -> global (fp32), dK and dQ times the softmax scale
@@ -388,35 +450,33 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             ++n_items;
             if (!ok) break;
             tc_fence_after_sync();
-            const bool store = kDq ? row_ok : outer_row < it.len;
-            const int32_t out_head = it.head;
             const int32_t out_heads = kDq ? p.num_q_heads : p.num_kv_heads;
-            const int64_t out_off = (static_cast<int64_t>(it.tok0 + outer_row) * out_heads + out_head) * D;
+            const int64_t out_off = (static_cast<int64_t>(it.tok0 + outer_row) * out_heads + it.head) * D;
+            // dK/dV: one warp group per accumulator; dQ: the groups split the columns of the one accumulator
+            const uint32_t acc_col = kDq ? 2 * kTile + D + grp * (D / 2) : 2 * kTile + grp * D;
+            float* dst = (kDq ? p.dq + grp * (D / 2) : (grp == 0 ? p.dv : p.dk)) + out_off;
+            const float mul = (kDq || grp == 1) ? p.scale : 1.f;
+            const bool add = !kDq && p.accumulate != 0;
+            constexpr int kChunks = (kDq ? D / 2 : D) / 32;
 #pragma unroll 1
-            for (int which = kDq ? 1 : 0; which < 2; ++which) {
-                float* dst = (which == 0 ? p.dv : (kDq ? p.dq : p.dk)) + out_off;
-                const float mul = which == 0 ? 1.f : p.scale;
-                const bool add = !kDq && p.accumulate != 0;
-#pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t a[32];
-                    tmem_ld32(tmem_base + 2 * kTile + which * D + c * 32 + lane_addr, a);
-                    tmem_ld_wait();
-                    if (store) {
+            for (int c = 0; c < kChunks; ++c) {
+                uint32_t a[32];
+                tmem_ld32(tmem_base + acc_col + c * 32 + lane_addr, a);
+                tmem_ld_wait();
+                if (row_ok) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            float4 v = make_float4(__uint_as_float(a[i]) * mul, __uint_as_float(a[i + 1]) * mul,
-                                                   __uint_as_float(a[i + 2]) * mul, __uint_as_float(a[i + 3]) * mul);
-                            float4* q4 = reinterpret_cast<float4*>(dst + c * 32 + i);
-                            if (add) {
-                                const float4 old = *q4;
-                                v.x += old.x;
-                                v.y += old.y;
-                                v.z += old.z;
-                                v.w += old.w;
-                            }
-                            *q4 = v;
+                    for (int i = 0; i < 32; i += 4) {
+                        float4 v = make_float4(__uint_as_float(a[i]) * mul, __uint_as_float(a[i + 1]) * mul,
+                                               __uint_as_float(a[i + 2]) * mul, __uint_as_float(a[i + 3]) * mul);
+                        float4* q4 = reinterpret_cast<float4*>(dst + c * 32 + i);
+                        if (add) {
+                            const float4 old = *q4;
+                            v.x += old.x;
+                            v.y += old.y;
+                            v.z += old.z;
+                            v.w += old.w;
                         }
+                        *q4 = v;
                     }
                 }
             }
