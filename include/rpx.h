@@ -25,9 +25,12 @@
  *     contiguous (stride head_dim) and a caller-given token stride in ELEMENTS.  Sequence s owns
  *     tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (int32, device, batch+1 entries, cu_seqlens[0]=0).
  *   - Query head h reads KV head h / (num_q_heads / num_kv_heads).
- *   - Element types: RPX_BF16 tensors are bfloat16; RPX_F32 tensors are float32 and are rounded
- *     to bf16 (nearest-even) in a pre-pass into the workspace, after which the same bf16
- *     tensor-core kernels run; outputs then come back as float32.  The KV cache is always bf16.
+ *   - Element types: RPX_BF16 tensors are bfloat16.  RPX_F32 tensors are float32 and exist for checking the
+ *     method against an unrounded reference, not for throughput: the attention calls then run an fp32 CUDA-core
+ *     kernel (q, the call's own k, v and every product stay fp32; out is float32), and the LM-head calls round
+ *     hidden and w_vocab to bf16 (nearest-even) in a pre-pass into the workspace before the tensor-core kernel.
+ *     The KV cache is always bf16: an RPX_F32 prefix pass stores K and V rounded to nearest-even, and a later
+ *     suffix or chunk pass reads those rounded values, as the bf16 path does.
  *   - Host-checkable problems (NULL pointer, head counts, head_dim, block size, alignment,
  *     strides, workspace size, device architecture) return a negative status BEFORE any launch.
  *     Problems only visible on the device (a kernel-side wait that ran out, an out-of-range

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 _CSRC = os.path.join(_HERE, "csrc")
 _OUT = os.path.join(_HERE, "librpx.so")
-SOURCES = ["rpx_api.cu", "rpx_host.cu", "rpx_logprobs.cu", "rpx_logprobs_bwd.cu", "rpx_attn.cu", "rpx_attn_bwd.cu"]
+SOURCES = ["rpx_api.cu", "rpx_host.cu", "rpx_logprobs.cu", "rpx_logprobs_bwd.cu", "rpx_attn.cu", "rpx_attn_bwd.cu", "rpx_attn_f32.cu"]
 
 
 def _nvcc() -> str:

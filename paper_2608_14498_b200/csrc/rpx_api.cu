@@ -22,18 +22,13 @@ rpx_status_t check_attn_desc(const rpx_attn_desc_t* d) {
     return RPX_OK;
 }
 
-// Layout: [work-item counter, kWsAlign bytes][RPX_F32 only: bf16 copies of q, k, v][suffix passes small enough
-// to be split over the cached prefix: split-KV partials]
-size_t attn_cast_workspace(const rpx_attn_desc_t* d, int64_t tokens) {
-    if (d->dtype != RPX_F32) return 0;
-    const size_t qb = align_up(static_cast<size_t>(tokens) * d->num_q_heads * d->head_dim * 2, kWsAlign);
-    const size_t kb = align_up(static_cast<size_t>(tokens) * d->num_kv_heads * d->head_dim * 2, kWsAlign);
-    return qb + 2 * kb;
-}
+// Layout: [work-item counter, kWsAlign bytes][suffix passes small enough to be split over the cached prefix:
+// split-KV partials].  The RPX_F32 path keeps nothing there, but asks for the counter's piece all the same so that a
+// caller's workspace handling does not depend on the element type.
 size_t attn_workspace(const rpx_attn_desc_t* d, int64_t tokens, bool is_suffix) {
     if (d == nullptr || tokens <= 0) return 0;
-    return kWsAlign + attn_cast_workspace(d, tokens) +
-           (is_suffix ? attn_split_workspace(tokens, d->num_q_heads, d->head_dim) : 0);
+    if (d->dtype == RPX_F32) return kWsAlign;
+    return kWsAlign + (is_suffix ? attn_split_workspace(tokens, d->num_q_heads, d->head_dim) : 0);
 }
 
 rpx_status_t check_cache(const rpx_kv_cache_t* c, int32_t batch) {
@@ -83,23 +78,6 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.q_tok_stride = q_tok_stride;
     a.k_tok_stride = k_tok_stride;
     a.v_tok_stride = v_tok_stride;
-    if (desc->dtype == RPX_F32) {
-        uint8_t* ws = static_cast<uint8_t*>(workspace) + kWsAlign;
-        const size_t qb = align_up(static_cast<size_t>(total_tokens) * q_row * 2, kWsAlign);
-        const size_t kb = align_up(static_cast<size_t>(total_tokens) * kv_row * 2, kWsAlign);
-        auto* qh = reinterpret_cast<__nv_bfloat16_raw*>(ws);
-        auto* kh = reinterpret_cast<__nv_bfloat16_raw*>(ws + qb);
-        auto* vh = reinterpret_cast<__nv_bfloat16_raw*>(ws + qb + kb);
-        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(q), q_tok_stride, qh, total_tokens, q_row, stream)) return rc;
-        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(k), k_tok_stride, kh, total_tokens, kv_row, stream)) return rc;
-        if (rpx_status_t rc = launch_cast_f32_bf16(static_cast<const float*>(v), v_tok_stride, vh, total_tokens, kv_row, stream)) return rc;
-        a.q = qh;
-        a.k = kh;
-        a.v = vh;
-        a.q_tok_stride = q_row;
-        a.k_tok_stride = kv_row;
-        a.v_tok_stride = kv_row;
-    }
     a.cu_seqlens = cu_seqlens;
     a.prefix_lens = is_suffix ? prefix_lens : nullptr;
     a.batch = batch;
@@ -108,14 +86,16 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
     a.max_prefix_len = max_prefix_len;
     a.cache = cache;
     a.item_counter = static_cast<uint32_t*>(workspace);
-    if (is_suffix && attn_split_workspace(total_tokens, desc->num_q_heads, desc->head_dim) > 0)
-        a.split_ws = static_cast<uint8_t*>(workspace) + kWsAlign + attn_cast_workspace(desc, total_tokens);
+    if (is_suffix && desc->dtype != RPX_F32 && attn_split_workspace(total_tokens, desc->num_q_heads, desc->head_dim) > 0)
+        a.split_ws = static_cast<uint8_t*>(workspace) + kWsAlign;
     a.append_cache = is_suffix && append_cache;
     a.out = out;
     a.out_f32 = desc->dtype == RPX_F32;
     a.lse = lse;
     a.device_status = device_status;
     a.stream = stream;
+    // fp32 tensors take the fp32 CUDA-core path; out is then float32 and 16-byte alignment is all the tensors need
+    if (desc->dtype == RPX_F32) return launch_attention_f32(a);
     return launch_attention(a);
 }
 

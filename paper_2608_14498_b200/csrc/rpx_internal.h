@@ -47,6 +47,8 @@ struct AttnArgs {
     cudaStream_t stream;
 };
 rpx_status_t launch_attention(const AttnArgs& a);
+// RPX_F32: q, k, v are float32 (strides in elements), out is float32; the cache stays bf16.
+rpx_status_t launch_attention_f32(const AttnArgs& a);
 // Split-KV workspace of a suffix pass over `tokens` query tokens: arrival counters, (max, sum) pairs and fp32
 // partial rows for up to 4 ranges; 0 when the pass is too large to ever be split.
 size_t attn_split_workspace(int64_t tokens, int32_t num_q_heads, int32_t head_dim);

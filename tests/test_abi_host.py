@@ -51,15 +51,17 @@ def test_sm_budget_is_host_state_with_validation(lib):
 
 
 def test_workspace_arithmetic(lib):
-    # every attention call keeps its work-item counter in the first 256 bytes; fp32 calls add bf16 copies of q, k, v
+    # every attention call keeps its work-item counter in the first 256 bytes; fp32 calls (CUDA-core path) use nothing
+    # of it but ask for the same piece
     assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 32768) == 256
     assert B.prefix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 0) == 0
     need = B.prefix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 256)
-    assert need == 256 + 256 * 4 * 64 * 2 + 2 * 256 * 2 * 64 * 2
+    assert need == 256
     # a suffix pass small enough to be split over the cached prefix also gets room for the partials of 4 ranges:
     # arrival counters, (max, sum) pairs and fp32 rows per (token, head)
     split = 512 + 4 * 128 * 8 + 4 * 128 * 64 * 4
-    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 256 + 32 * 8 * 64 * 2 + split
+    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_BF16, 32) == 256 + split
+    assert B.suffix_attn_workspace_bytes(4, 2, 64, B.RPX_F32, 32) == 256
     assert B.suffix_attn_workspace_bytes(28, 4, 128, B.RPX_BF16, 113377) == 256  # too many rows to be worth splitting
     # 152064 columns = 594 tiles of 256; one float4 per (chunk, row): 38 chunks of 16 tiles up to 191 row
     # tiles of 128 rows, 75 chunks of 8 tiles from 192 row tiles on

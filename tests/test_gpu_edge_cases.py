@@ -104,18 +104,11 @@ def test_strided_fp32_inputs(cuda_device):
     assert o.dtype == torch.float32
     rows = oracle.all_rows(wl.cu_full, 4)
     got, got_l = o.double().cpu().numpy().reshape(-1, 64), lse.double().cpu().numpy().reshape(-1)
-    # fp32 tensors are rounded to bf16 before the tensor core.  Against the oracle fed the same
-    # rounded inputs only the kernel's own error is left (<= 1e-2 as for bf16 configs) ...
-    rb = lambda a: wk.f32_to_bf16_bits(a).reshape(a.shape)
-    ref_b, ref_bl = oracle.attn_rows(rb(wl.q), rb(wl.k), rb(wl.v), wl.cu_full, rows)
-    assert np.abs(got - ref_b).max() <= 1e-2
-    assert np.abs(got_l - ref_bl).max() <= 2e-3
-    # ... and against the unrounded inputs the input rounding adds up to 2^-9 per operand on values
-    # of magnitude <= 4.5 here: 3 * 4.5 * 2^-9 = 2.6e-2 (observed about half of that)
+    # fp32 tensors take the fp32 CUDA-core path: nothing is rounded in a prefix pass, so the unrounded oracle is met
+    # to fp32 accuracy (sums of <= 70 products of magnitude <= 20, exp2 to 2^-22)
     ref, ref_l = oracle.attn_rows(wl.q, wl.k, wl.v, wl.cu_full, rows)
-    print("fp32-input attention error vs unrounded oracle:", np.abs(got - ref).max())
-    assert np.abs(got - ref).max() <= 2.6e-2
-    assert np.abs(got_l - ref_l).max() <= 2.6e-2
+    assert np.abs(got - ref).max() <= 2e-5
+    assert np.abs(got_l - ref_l).max() <= 2e-5
 
 
 def test_a_sequence_longer_than_the_callers_bound_is_reported(cuda_device):

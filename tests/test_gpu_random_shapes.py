@@ -46,9 +46,17 @@ def test_random_batch_matches_the_oracle(cuda_device, case):
     rows = oracle.all_rows(wl.cu_full, cfg.num_q_heads)
     if cfg.dtype == "bf16":
         T.check_rows(wl, out, lse, rows)
-    else:  # fp32 inputs are rounded to bf16 first: compare with the oracle on the rounded inputs
-        rb = lambda a: wk.f32_to_bf16_bits(a).reshape(a.shape)
-        T.check_rows(wl, out, lse, rows, inputs=(rb(wl.q), rb(wl.k), rb(wl.v)))
+    else:
+        # fp32 tensors: against the UNROUNDED oracle.  The only rounding left is that of the prompt's K/V in the
+        # bf16 cache the suffix pass reads, so the prompt rows match to fp32 accuracy and the response rows stay
+        # inside the bound of the bf16 configs.
+        T.check_rows(wl, out, lse, rows, lse_tol=1e-2)
+        pre = rows[rows[:, 1] < wl.prompt_lens[rows[:, 0]]]
+        if pre.shape[0]:
+            ref_o, ref_l = oracle.attn_rows(wl.q, wl.k, wl.v, wl.cu_full, pre)
+            tok = wl.cu_full[pre[:, 0]].astype(np.int64) + pre[:, 1]
+            assert np.abs(out[tok, pre[:, 2]] - ref_o).max() <= 5e-5
+            assert np.abs(lse[tok, pre[:, 2]] - ref_l).max() <= 5e-5
     T.check_cache(wl, kc, vc)
     # LM head on the prompt rows and on the response rows, concatenated = the full-sequence values
     status = torch.zeros(1, dtype=torch.int32, device=dev)
