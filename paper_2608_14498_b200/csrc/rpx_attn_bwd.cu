@@ -42,7 +42,7 @@ namespace rpx {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kStages = 2;   // inner (Y1, Y2) pairs in flight
+constexpr int kStages = 4;   // half inner tiles (64 rows of Y1 and of Y2) in flight: two steps of data, released a half at a time (a fifth stage measured no faster)
 constexpr int kThreads = 320;
 constexpr int kHalf = 64;    // inner rows per half step
 constexpr uint32_t kTmemCols = 512;
@@ -62,7 +62,7 @@ struct Ctl {
     uint32_t abort_flag;
     uint32_t drain_flag;
     uint32_t data_error;
-    float vec[kStages][2][kTile]; // kDq = false: (-lse * log2 e or -inf, -D) of the inner query tile, per stage
+    float vec[kStages][2][kHalf]; // kDq = false: (-lse * log2 e or -inf, -D) of the stage's 64 inner query rows
 };
 
 template <int D>
@@ -71,8 +71,11 @@ struct Layout {
     static constexpr int kHalfBytes = kTile * 128;
     static constexpr int kTileBytes = kHalves * kHalfBytes;
     static constexpr int kOuterOff = 0;                                  // X1, X2
-    static constexpr int kInnerOff = 2 * kTileBytes;                     // kStages x (Y1, Y2)
-    static constexpr int kCtlOff = kInnerOff + kStages * 2 * kTileBytes;
+    static constexpr int kInnerOff = 2 * kTileBytes;                     // kStages x (Y1 half, Y2 half)
+    static constexpr int kBlockBytes = kHalf * 128;                      // one [64 rows][64 bf16] swizzled block of a half
+    static constexpr int kHalfTileBytes = kHalves * kBlockBytes;         // 64 rows of one inner tile
+    static constexpr int kStageBytes = 2 * kHalfTileBytes;
+    static constexpr int kCtlOff = kInnerOff + kStages * kStageBytes;
     static constexpr size_t kSmemBytes = kCtlOff + sizeof(Ctl);
 };
 
@@ -125,6 +128,27 @@ __device__ __forceinline__ int32_t item_of_round(int32_t rnd) {
     return rnd * g + ((rnd & 1) ? g - 1 - b : b);
 }
 
+// Eight K=16 steps of D = A * B: A's two 64-element K blocks lie 16 KiB (1024 units) apart (a 128-row tile), B's
+// 8 KiB (512 units) apart (a 64-row half tile).
+__device__ __forceinline__ void umma_ss_k128_half_b(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+#define RPX_UMMA_SS_STEP_AB(aoff, boff)                                        \
+    "add.s64 da, %1, " #aoff ";\n"                                             \
+    "add.s64 db, %2, " #boff ";\n"                                             \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n"
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 pf, %3, %3;\n"
+        "setp.eq.b32 pt, %3, %3;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n" RPX_UMMA_SS_STEP_AB(2, 2) RPX_UMMA_SS_STEP_AB(4, 4)
+            RPX_UMMA_SS_STEP_AB(6, 6) RPX_UMMA_SS_STEP_AB(1024, 512) RPX_UMMA_SS_STEP_AB(1026, 514)
+                RPX_UMMA_SS_STEP_AB(1028, 516) RPX_UMMA_SS_STEP_AB(1030, 518) "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc)
+        : "memory");
+#undef RPX_UMMA_SS_STEP_AB
+}
+
 template <bool kDq>
 __device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
     Item it;
@@ -165,8 +189,10 @@ __device__ __forceinline__ Item decode_item(const Params& p, int32_t idx) {
 
 template <int D, bool kDq>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do, const Params p) {
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_x1, const __grid_constant__ CUtensorMap tmap_x2,
+                const __grid_constant__ CUtensorMap tmap_y1, const __grid_constant__ CUtensorMap tmap_y2, const Params p) {
+    // x1, x2: the outer tiles' tensors (K, V for dK/dV; Q, dO for dQ), boxes of 128 rows; y1, y2: the inner tiles'
+    // (Q, dO; K, V), boxes of 64 rows
     using L = Layout<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     if ((smem_u32(smem) & 1023u) != 0u) {
@@ -206,10 +232,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
     // TMEM columns: T1 at 0, T2 at 128, accumulator a at 256, accumulator b at 256 + D
-    const CUtensorMap* map_x1 = kDq ? &tmap_q : &tmap_k;
-    const CUtensorMap* map_x2 = kDq ? &tmap_do : &tmap_v;
-    const CUtensorMap* map_y1 = kDq ? &tmap_k : &tmap_q;
-    const CUtensorMap* map_y2 = kDq ? &tmap_v : &tmap_do;
+    const CUtensorMap *map_x1 = &tmap_x1, *map_x2 = &tmap_x2, *map_y1 = &tmap_y1, *map_y2 = &tmap_y2;
 
     if (warp == 0) {
         // =========================================================== producer warp
@@ -236,18 +259,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             for (int32_t hh = 0; ok && hh < it.n_heads; ++hh) {
                 const int32_t qh = kDq ? it.head : it.head * p.group + hh;  // the query head of this inner run
-                for (int32_t in = it.in_lo; ok && in <= it.in_hi; ++in, ++n_in) {
+                for (int32_t in2 = 2 * it.in_lo; ok && in2 <= 2 * it.in_hi + 1; ++in2, ++n_in) {
+                    const int32_t in = in2 >> 1, h = in2 & 1;  // n_in counts half tiles here
                     const uint32_t stage = n_in % kStages, phase = (n_in / kStages) & 1u;
                     if (!mbar_wait(&ctl->in_empty[stage], phase ^ 1u, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    uint8_t* y1 = smem + L::kInnerOff + stage * 2 * L::kTileBytes;
-                    uint8_t* y2 = y1 + L::kTileBytes;
+                    uint8_t* y1 = smem + L::kInnerOff + stage * L::kStageBytes;
+                    uint8_t* y2 = y1 + L::kHalfTileBytes;
                     if (!kDq) {
                         // -lse (in log2 units) and -D of the inner query tile, for the element-wise warps
-                        for (int32_t r = lane; r < kTile; r += 32) {
-                            const int32_t qr = in * kTile + r;
+                        for (int32_t r = lane; r < kHalf; r += 32) {
+                            const int32_t qr = in * kTile + h * kHalf + r;
                             float l2 = -CUDART_INF_F, dd = 0.f;  // a row that takes no part: P = 2^(-inf) = 0, dS = 0
                             if (qr >= it.qb && qr < it.qe) {
                                 const int64_t rh = static_cast<int64_t>(it.tok0 + qr) * p.num_q_heads + qh;
@@ -260,12 +284,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         __syncwarp();
                     }
                     if (lane == 0) {
-                        mbar_arrive_expect_tx(&ctl->in_full[stage], 2 * L::kTileBytes);
+                        mbar_arrive_expect_tx(&ctl->in_full[stage], L::kStageBytes);
                         for (int hf = 0; hf < L::kHalves; ++hf) {
-                            tma_load_3d(y1 + hf * L::kHalfBytes, map_y1, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
-                                        it.tok0 + in * kTile);
-                            tma_load_3d(y2 + hf * L::kHalfBytes, map_y2, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
-                                        it.tok0 + in * kTile);
+                            tma_load_3d(y1 + hf * L::kBlockBytes, map_y1, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
+                                        it.tok0 + in * kTile + h * kHalf);
+                            tma_load_3d(y2 + hf * L::kBlockBytes, map_y2, &ctl->in_full[stage], hf * 64, kDq ? kv_head : qh,
+                                        it.tok0 + in * kTile + h * kHalf);
                         }
                     }
                     __syncwarp();
@@ -284,19 +308,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (elect_one()) {
             constexpr uint32_t idesc_t = make_idesc_bf16(kTile, kHalf, false, false);
             constexpr uint32_t idesc_acc = make_idesc_bf16(kTile, D, false, true);
-            constexpr uint32_t kHalfUnits = kHalf * 128 / 16;  // 64 rows of 128 bytes, in descriptor units of 16 bytes
             const uint32_t outer_addr = smem_u32(smem + L::kOuterOff);
             const uint32_t inner_addr = smem_u32(smem + L::kInnerOff);
             const uint64_t x1_desc = make_smem_desc_sw128(outer_addr, 16, 1024);
             const uint64_t x2_desc = make_smem_desc_sw128(outer_addr + L::kTileBytes, 16, 1024);
             // T1 = X1 Y1^T and T2 = X2 Y2^T for the inner rows 64 h .. 64 h + 63 of the pair in `stage`
             auto issue_t = [&](uint32_t stage, int h) {
-                const uint32_t y1_addr = inner_addr + stage * 2 * L::kTileBytes;
-                const uint64_t y1_k = make_smem_desc_sw128(y1_addr, 16, 1024) + h * kHalfUnits;
-                const uint64_t y2_k = make_smem_desc_sw128(y1_addr + L::kTileBytes, 16, 1024) + h * kHalfUnits;
+                const uint32_t y1_addr = inner_addr + stage * L::kStageBytes;
+                const uint64_t y1_k = make_smem_desc_sw128(y1_addr, 16, 1024);
+                const uint64_t y2_k = make_smem_desc_sw128(y1_addr + L::kHalfTileBytes, 16, 1024);
                 if (D == 128) {
-                    umma_ss_k128_overwrite(tmem_base + h * kHalf, x1_desc, y1_k, idesc_t);
-                    umma_ss_k128_overwrite(tmem_base + kTile + h * kHalf, x2_desc, y2_k, idesc_t);
+                    umma_ss_k128_half_b(tmem_base + h * kHalf, x1_desc, y1_k, idesc_t);
+                    umma_ss_k128_half_b(tmem_base + kTile + h * kHalf, x2_desc, y2_k, idesc_t);
                 } else {
                     umma_ss_k64_overwrite(tmem_base + h * kHalf, x1_desc, y1_k, idesc_t);
                     umma_ss_k64_overwrite(tmem_base + kTile + h * kHalf, x2_desc, y2_k, idesc_t);
@@ -312,19 +335,22 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 // the accumulators still hold the previous item's result until its epilogue has read them
                 if (ok && n_items > 0) ok = mbar_wait(&ctl->acc_free, (n_items - 1) & 1u, abort_flag);
                 const int32_t steps = it.n_heads * (it.in_hi - it.in_lo + 1);
-                if (ok) ok = mbar_wait(&ctl->in_full[n_in % kStages], (n_in / kStages) & 1u, abort_flag);
-                if (ok) {
-                    tc_fence_after_sync();
-                    issue_t(n_in % kStages, 0);
-                    issue_t(n_in % kStages, 1);
-                    if (steps == 1) umma_commit(&ctl->outer_empty);
+                // n_in counts steps; the half tile (step n, half h) is the ring's entry 2 n + h
+                for (int h = 0; ok && h < 2; ++h) {
+                    const uint32_t e = 2 * n_in + h;
+                    ok = mbar_wait(&ctl->in_full[e % kStages], (e / kStages) & 1u, abort_flag);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        issue_t(e % kStages, h);
+                    }
                 }
+                if (ok && steps == 1) umma_commit(&ctl->outer_empty);
                 for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
-                    const uint32_t stage = n_in % kStages;
-                    const uint32_t y1_addr = inner_addr + stage * 2 * L::kTileBytes;
-                    const uint64_t y1_mn = make_smem_desc_sw128(y1_addr, L::kHalfBytes, 1024);                  // MN-major
-                    const uint64_t y2_mn = make_smem_desc_sw128(y1_addr + L::kTileBytes, L::kHalfBytes, 1024);
                     for (int h = 0; ok && h < 2; ++h) {
+                        const uint32_t stage = (2 * n_in + h) % kStages;
+                        const uint32_t y1_addr = inner_addr + stage * L::kStageBytes;
+                        const uint64_t y1_mn = make_smem_desc_sw128(y1_addr, L::kBlockBytes, 1024);              // MN-major
+                        const uint64_t y2_mn = make_smem_desc_sw128(y1_addr + L::kHalfTileBytes, L::kBlockBytes, 1024);
                         if (!mbar_wait(&ctl->e_ready[h], n_in & 1u, abort_flag)) {
                             ok = false;
                             break;
@@ -333,15 +359,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         // accumulate over the 64 inner rows of the half: a += P Y2 (dV; not for dQ), b += dS Y1 (dK or dQ)
                         const uint32_t acc = (s != 0 || h != 0) ? 1u : 0u;
                         if (!kDq)
-                            umma_ts_k64_split(tmem_base + 2 * kTile, tmem_base + h * kHalf, y2_mn + h * kHalfUnits, idesc_acc, acc);
-                        umma_ts_k64_split(tmem_base + 2 * kTile + D, tmem_base + kTile + h * kHalf, y1_mn + h * kHalfUnits,
-                                          idesc_acc, acc);
-                        if (h == 1) umma_commit(&ctl->in_empty[stage]);
+                            umma_ts_k64_split(tmem_base + 2 * kTile, tmem_base + h * kHalf, y2_mn, idesc_acc, acc);
+                        umma_ts_k64_split(tmem_base + 2 * kTile + D, tmem_base + kTile + h * kHalf, y1_mn, idesc_acc, acc);
+                        umma_commit(&ctl->in_empty[stage]);
                         if (s + 1 < steps) {
                             // the next step's T of this half, in order behind the accumulate MMAs that read P / dS from
                             // the same columns
-                            const uint32_t nstage = (n_in + 1) % kStages;
-                            if (h == 0 && !mbar_wait(&ctl->in_full[nstage], ((n_in + 1) / kStages) & 1u, abort_flag)) {
+                            const uint32_t ne = 2 * (n_in + 1) + h, nstage = ne % kStages;
+                            if (!mbar_wait(&ctl->in_full[nstage], (ne / kStages) & 1u, abort_flag)) {
                                 ok = false;
                                 break;
                             }
@@ -387,15 +412,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const int32_t n_inner = it.in_hi - it.in_lo + 1;
             const int32_t steps = it.n_heads * n_inner;
             for (int32_t s = 0; ok && s < steps; ++s, ++n_in) {
-                const uint32_t stage = n_in % kStages;
                 const int32_t in = it.in_lo + s % n_inner;
                 const bool diagonal = in == it.tile;
-                // the producer's lse / D vectors of this stage are visible once the stage's barrier has completed
-                if (!kDq && !mbar_wait(&ctl->in_full[stage], (n_in / kStages) & 1u, abort_flag)) {
-                    ok = false;
-                    break;
-                }
                 for (int h = 0; h < 2; ++h) {
+                    const uint32_t e = 2 * n_in + h, stage = e % kStages;
+                    // the producer's lse / D vectors of this stage are visible once the stage's barrier has completed
+                    if (!kDq && !mbar_wait(&ctl->in_full[stage], (e / kStages) & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
                     if (!mbar_wait(&ctl->t_full[h], n_in & 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -414,8 +439,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             nl2 = nl2_row;
                             nd = nd_row;
                         } else {
-                            const float2 lv = *reinterpret_cast<const float2*>(&ctl->vec[stage][0][col + i]);
-                            const float2 dv2 = *reinterpret_cast<const float2*>(&ctl->vec[stage][1][col + i]);
+                            const float2 lv = *reinterpret_cast<const float2*>(&ctl->vec[stage][0][grp * 32 + i]);
+                            const float2 dv2 = *reinterpret_cast<const float2*>(&ctl->vec[stage][1][grp * 32 + i]);
                             nl2 = f2_pack(lv.x, lv.y);
                             nd = f2_pack(dv2.x, dv2.y);
                         }
@@ -528,22 +553,25 @@ __global__ void attn_bwd_zero_kernel(float* __restrict__ a, float* __restrict__ 
 template <int D>
 rpx_status_t launch_d(const AttnBwdArgs& a) {
     using L = Layout<D>;
-    CUtensorMap tq, tk, tv, tdo;
+    // every tensor twice: boxes of 128 rows where it is the outer tile, of 64 rows where it is streamed as inner halves
+    CUtensorMap tq[2], tk[2], tv[2], tdo[2];
     const uint64_t tokens = static_cast<uint64_t>(a.total_tokens);
-    const uint32_t box[3] = {64, 1, kTile};
-    {
-        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_q_heads), tokens};
-        const uint64_t qs[2] = {D * 2ull, static_cast<uint64_t>(a.q_tok_stride) * 2};
-        const uint64_t os[2] = {D * 2ull, static_cast<uint64_t>(a.num_q_heads) * D * 2ull};
-        if (rpx_status_t rc = encode_tmap_bf16(&tq, a.q, 3, dims, qs, box)) return rc;
-        if (rpx_status_t rc = encode_tmap_bf16(&tdo, a.dout, 3, dims, os, box)) return rc;
-    }
-    {
-        const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_kv_heads), tokens};
-        const uint64_t ks[2] = {D * 2ull, static_cast<uint64_t>(a.k_tok_stride) * 2};
-        const uint64_t vs[2] = {D * 2ull, static_cast<uint64_t>(a.v_tok_stride) * 2};
-        if (rpx_status_t rc = encode_tmap_bf16(&tk, a.k, 3, dims, ks, box)) return rc;
-        if (rpx_status_t rc = encode_tmap_bf16(&tv, a.v, 3, dims, vs, box)) return rc;
+    for (int m = 0; m < 2; ++m) {
+        const uint32_t box[3] = {64, 1, m == 0 ? static_cast<uint32_t>(kTile) : static_cast<uint32_t>(kHalf)};
+        {
+            const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_q_heads), tokens};
+            const uint64_t qs[2] = {D * 2ull, static_cast<uint64_t>(a.q_tok_stride) * 2};
+            const uint64_t os[2] = {D * 2ull, static_cast<uint64_t>(a.num_q_heads) * D * 2ull};
+            if (rpx_status_t rc = encode_tmap_bf16(&tq[m], a.q, 3, dims, qs, box)) return rc;
+            if (rpx_status_t rc = encode_tmap_bf16(&tdo[m], a.dout, 3, dims, os, box)) return rc;
+        }
+        {
+            const uint64_t dims[3] = {D, static_cast<uint64_t>(a.num_kv_heads), tokens};
+            const uint64_t ks[2] = {D * 2ull, static_cast<uint64_t>(a.k_tok_stride) * 2};
+            const uint64_t vs[2] = {D * 2ull, static_cast<uint64_t>(a.v_tok_stride) * 2};
+            if (rpx_status_t rc = encode_tmap_bf16(&tk[m], a.k, 3, dims, ks, box)) return rc;
+            if (rpx_status_t rc = encode_tmap_bf16(&tv[m], a.v, 3, dims, vs, box)) return rc;
+        }
     }
     int sms = sm_count();
     if (sms <= 0) return RPX_ERR_CUDA;
@@ -591,7 +619,7 @@ rpx_status_t launch_d(const AttnBwdArgs& a) {
         if (items > INT32_MAX) return RPX_ERR_SHAPE;
         p.n_items = static_cast<int32_t>(items);
         const unsigned grid = static_cast<unsigned>(items < sms ? items : sms);
-        attn_bwd_kernel<D, false><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tdo, p);
+        attn_bwd_kernel<D, false><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tk[0], tv[0], tq[1], tdo[1], p);
         if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
     }
     {
@@ -599,7 +627,7 @@ rpx_status_t launch_d(const AttnBwdArgs& a) {
         if (items > INT32_MAX) return RPX_ERR_SHAPE;
         p.n_items = static_cast<int32_t>(items);
         const unsigned grid = static_cast<unsigned>(items < sms ? items : sms);
-        attn_bwd_kernel<D, true><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tdo, p);
+        attn_bwd_kernel<D, true><<<grid, kThreads, L::kSmemBytes, a.stream>>>(tq[0], tdo[0], tk[1], tv[1], p);
         if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
     }
     return RPX_OK;
