@@ -179,3 +179,32 @@ def test_sequence_offsets_that_leave_the_tensors_are_reported(cuda_device):
     _close(dq[:200], rq, "dq")
     _close(dk[:200], rk, "dk")
     assert float(dq[200:].abs().max()) == 0.0 and float(dk[200:].abs().max()) == 0.0
+
+
+def test_c2_at_full_size_against_the_oracle_on_one_kv_group(cuda_device):
+    """The benchmark's backward workload (C2: 8 whole sequences of 4352 tokens, 28 query / 4 KV heads, head_dim 128)
+    through the same call the benchmark times; the oracle differentiates one (sequence, KV head) slice - attention
+    and its gradients are independent per sequence and KV group, so the slice is a complete problem."""
+    dev = cuda_device
+    cfg = wk.CONFIGS["C2"]
+    wl = wk.make_workload(cfg, seed=0, lm=False)
+    dout = wk.make_workload(cfg, seed=1, lm=False).q
+    tq, tk, tv, tdo, tcu = (to_device(x, dev) for x in (wl.q, wl.k, wl.v, dout, wl.cu_full))
+    lens = (wl.prompt_lens + wl.response_lens).astype(np.int64)
+    max_len = int(lens.max())
+    out, lse = _forward(dev, tq, tk, tv, tcu, max_len)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    dq, dk, dv = rpx.attn_backward(tq, tk, tv, out, tdo, lse, tcu, max_len, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    seq, g = 5, 2
+    group = cfg.num_q_heads // cfg.num_kv_heads
+    a, b = int(wl.cu_full[seq]), int(wl.cu_full[seq + 1])
+    hs = slice(g * group, (g + 1) * group)
+    cu1 = np.array([0, b - a], dtype=np.int32)
+    do64 = wk.bf16_bits_to_f32(dout[a:b, hs]).reshape(b - a, group, cfg.head_dim).astype(np.float64)
+    rq, rk, rv = oracle.attn_backward(np.ascontiguousarray(wl.q[a:b, hs]), np.ascontiguousarray(wl.k[a:b, g:g + 1]),
+                                      np.ascontiguousarray(wl.v[a:b, g:g + 1]), cu1, do64)
+    _close(dq[a:b, hs], rq, "dq")
+    _close(dk[a:b, g:g + 1], rk, "dk")
+    _close(dv[a:b, g:g + 1], rv, "dv")
