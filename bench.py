@@ -3,6 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3]
     python bench.py --profile-case lm|lmbwd|prefix|suffix|attnbwd [--reps 3]      (small launches for profiler captures)
+    python bench.py --attn-alone [--reps 30]                             (attention passes of C2, C3, C4 timed alone)
 
 One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
 boundary-KV write), prefix log-probs, suffix attention over the cached KV, suffix log-probs.
@@ -587,6 +588,79 @@ def run_profile_case(args):
     print(f"profile case {case}: ok")
 
 
+def run_attn_alone(args):
+    """The attention passes alone, `reps` launches back to back per pass and config, with the clocks sampled during
+    each timed region: what the kernels do at the clock they reach when the LM head's power draw is not setting it.
+    One JSON line per config (C2, C3, C4): prefix pass (with cache write), suffix pass, TFLOP/s on the algorithmic
+    (causal) flops and fractions of the measured peaks."""
+    import torch
+
+    import paper_2608_14498_b200 as rpx
+
+    dev = torch.device("cuda", 0)
+    peaks = load_peaks()
+    try:
+        gpu_id = str(torch.cuda.get_device_properties(0).uuid)
+        gpu_id = gpu_id if gpu_id.startswith("GPU-") else "GPU-" + gpu_id
+    except Exception:
+        gpu_id = "0"
+
+    def t(a):
+        x = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return x.to(dev)
+
+    def timed(call):
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(gpu_id)
+        time.sleep(0.3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.mark()
+        e0.record()
+        for _ in range(args.reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        sampler.mark()
+        return e0.elapsed_time(e1) / args.reps, sampler.stop()
+
+    for name in ("C2", "C3", "C4"):
+        cfg = wk.CONFIGS[name]
+        wl = wk.make_workload(cfg, seed=0, lm=False)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        kc = torch.zeros((wl.num_blocks, cfg.num_kv_heads, 16, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+        cache = (kc, torch.zeros_like(kc), t(wl.block_table))
+        qp, kp, vp = (t(wl.prefix_pack(x)) for x in (wl.q, wl.k, wl.v))
+        qs, ks, vs = (t(wl.suffix_pack(x)) for x in (wl.q, wl.k, wl.v))
+        cu_p, cu_s, pl = t(wl.cu_prefix), t(wl.cu_suffix), t(wl.prompt_lens)
+        max_p, max_r = int(wl.prompt_lens.max()), int(wl.response_lens.max())
+        op, os_ = torch.empty_like(qp), torch.empty_like(qs)
+        ws_p = torch.empty(rpx.prefix_attn_workspace_bytes(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, 0, qp.shape[0]),
+                           dtype=torch.uint8, device=dev)
+        ws_s = torch.empty(rpx.suffix_attn_workspace_bytes(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, 0, qs.shape[0]),
+                           dtype=torch.uint8, device=dev)
+        ms_p, clk_p = timed(lambda: rpx.prefix_attn(qp, kp, vp, cu_p, max_p, cache=cache, out=op, workspace=ws_p,
+                                                    device_status=status))
+        ms_s, clk_s = timed(lambda: rpx.suffix_attn(qs, ks, vs, cu_s, pl, max_r, max_p, cache=cache, out=os_, workspace=ws_s,
+                                                    device_status=status))
+        if int(status.item()) != 0:
+            raise SystemExit(f"device status {int(status.item())}")
+        p64, r64 = wl.prompt_lens.astype(np.float64), wl.response_lens.astype(np.float64)
+        fl_p = float((4.0 * cfg.head_dim * cfg.num_q_heads * p64 * (p64 + 1) / 2).sum())
+        fl_s = float((4.0 * cfg.head_dim * cfg.num_q_heads * (r64 * p64 + r64 * (r64 + 1) / 2)).sum())
+        rec = {"workload": cfg.name, "reps": args.reps}
+        for key, ms, fl, clk in (("prefix_attn", ms_p, fl_p, clk_p), ("suffix_attn", ms_s, fl_s, clk_s)):
+            tf = fl / (ms * 1e-3) / 1e12
+            rec[key] = {"ms": ms, "tflops": tf,
+                        "frac_of_sustained_peak": tf / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+                        "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]), "frac_of_datasheet": tf / 2250.0,
+                        "clocks": clk}
+        print(json.dumps(rec), flush=True)
+        del qp, kp, vp, qs, ks, vs, op, os_, kc, cache
+        torch.cuda.empty_cache()
+
+
 def run_group(args):
     """Prompt groups (GRPO: N sampled responses per prompt).  Times one scoring pass with the prompt
     prefix computed once per group (cache rows aliased by the group's members) against the same
@@ -669,6 +743,7 @@ def main():
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
     ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
     ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix", "attnbwd"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--attn-alone", action="store_true", help="time the attention passes of C2, C3 and C4 alone (--reps launches each)")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of --impl reference")
@@ -682,6 +757,11 @@ def main():
     if args.profile_case:
         if rank == 0:
             run_profile_case(args)
+    elif args.attn_alone:
+        if rank == 0:
+            if args.reps < 10:
+                args.reps = 30
+            run_attn_alone(args)
     elif args.group > 0:
         if rank == 0:
             run_group(args)
