@@ -317,6 +317,7 @@ def measure_config(torch, dist, config, steps, warmup, rank, local_rank, world, 
                    "response_tokens": wl.n_suffix, "scored_tokens_per_gpu": wl.n_tokens, "q_heads": cfg.num_q_heads,
                    "kv_heads": cfg.num_kv_heads, "head_dim": cfg.head_dim, "hidden": cfg.hidden, "vocab": cfg.vocab,
                    "kv_block": 16, "parallelism": f"dp{world} (independent sequences per rank, no collective)",
+                   "lm_head_kernel": "CTA pairs (cta_group::2)" if rpx.get_lm_head_pairing() else "one CTA per tile",
                    "l2": f"no flush: per-step inputs (W_vocab {gb(wl.w.nbytes)}, hidden {gb(wl.hidden.nbytes)}, "
                          f"Q/K/V {gb(wl.q.nbytes + wl.k.nbytes + wl.v.nbytes)}) exceed the 126 MB L2",
                    "stands_in_for": cfg.stands_in_for},
@@ -743,6 +744,8 @@ def main():
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
     ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
     ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix", "attnbwd"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--lm-head-pairing", action="store_true",
+                    help="run the LM head's CTA-pair (cta_group::2) kernel instead of the single-CTA one")
     ap.add_argument("--attn-alone", action="store_true", help="time the attention passes of C2, C3 and C4 alone (--reps launches each)")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case after its warm-up launch")
     ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens the oracle scores for cpu_baseline (~10-20 s)")
@@ -754,6 +757,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.lm_head_pairing and args.impl != "reference":
+        import paper_2608_14498_b200 as rpx
+
+        rpx.set_lm_head_pairing(True)
     if args.profile_case:
         if rank == 0:
             run_profile_case(args)

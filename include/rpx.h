@@ -334,6 +334,16 @@ RPX_API rpx_status_t rpx_selftest_bounded_wait(int64_t limit_cycles, int32_t* de
 RPX_API rpx_status_t rpx_set_sm_budget(int32_t sms);
 RPX_API int32_t rpx_get_sm_budget(void);
 
+/*
+ * Which LM-head kernel later calls of this process use (rpx_token_logprobs, _entropy, _shard, _static): 0 = one
+ * CTA per 128 x 256 tile, != 0 = CTA pairs (a cluster of two CTAs per 256 x 256 tile, tcgen05 cta_group::2: each
+ * CTA loads its own 128 rows of hidden states and half of the W tile, the even CTA issues the MMAs for both).
+ * Results equal each other up to the order of fp32 partial sums (the partial records of a row do not depend on
+ * which kernel produced them; the split of the vocabulary into chunks is the same).  Host-only state.
+ */
+RPX_API rpx_status_t rpx_set_lm_head_pairing(int32_t on);
+RPX_API int32_t rpx_get_lm_head_pairing(void);
+
 /* Static string for a status code; never NULL. */
 RPX_API const char* rpx_status_string(rpx_status_t status);
 

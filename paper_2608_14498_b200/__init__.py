@@ -9,12 +9,14 @@ from .binding import (  # noqa: F401
     attn_backward,
     attn_backward_workspace_bytes,
     chunk_attn,
+    get_lm_head_pairing,
     get_sm_budget,
     library_path,
     load_library,
     prefix_attn,
     prefix_attn_workspace_bytes,
     selftest_bounded_wait,
+    set_lm_head_pairing,
     set_sm_budget,
     status_string,
     suffix_attn,

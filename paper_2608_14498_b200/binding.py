@@ -29,6 +29,8 @@ EXPORTS = (
     "rpx_token_logprobs_static",
     "rpx_token_logprobs_backward",
     "rpx_token_logprobs_backward_workspace_bytes",
+    "rpx_set_lm_head_pairing",
+    "rpx_get_lm_head_pairing",
     "rpx_attn_backward",
     "rpx_attn_backward_workspace_bytes",
     "rpx_prefix_attn_workspace_bytes",
@@ -125,6 +127,10 @@ def load_library():
     lib.rpx_set_sm_budget.argtypes = [i32]
     lib.rpx_get_sm_budget.restype = i32
     lib.rpx_get_sm_budget.argtypes = []
+    lib.rpx_set_lm_head_pairing.restype = i32
+    lib.rpx_set_lm_head_pairing.argtypes = [i32]
+    lib.rpx_get_lm_head_pairing.restype = i32
+    lib.rpx_get_lm_head_pairing.argtypes = []
     lib.rpx_status_string.restype = ctypes.c_char_p
     lib.rpx_status_string.argtypes = [i32]
     lib.rpx_version.restype = i32
@@ -252,6 +258,17 @@ def set_sm_budget(sms: int) -> None:
     rc = load_library().rpx_set_sm_budget(int(sms))
     if rc != 0:
         raise RpxError(rc, "rpx_set_sm_budget")
+
+
+def set_lm_head_pairing(on: bool) -> None:
+    """Process-wide choice of the LM-head kernel: CTA pairs (cta_group::2) when ``on``."""
+    rc = load_library().rpx_set_lm_head_pairing(1 if on else 0)
+    if rc != 0:
+        raise RpxError(rc, "rpx_set_lm_head_pairing")
+
+
+def get_lm_head_pairing() -> bool:
+    return bool(load_library().rpx_get_lm_head_pairing())
 
 
 def get_sm_budget() -> int:

@@ -386,6 +386,13 @@ rpx_status_t rpx_set_sm_budget(int32_t sms) {
 
 int32_t rpx_get_sm_budget(void) { return rpx::sm_budget(); }
 
+rpx_status_t rpx_set_lm_head_pairing(int32_t on) {
+    rpx::set_lm_head_pairing(on);
+    return RPX_OK;
+}
+
+int32_t rpx_get_lm_head_pairing(void) { return rpx::lm_head_pairing(); }
+
 int32_t rpx_version(void) { return 100; }
 
 }  // extern "C"

@@ -92,6 +92,9 @@ std::atomic<int> g_sm_budget{0};
 }
 int sm_budget() { return g_sm_budget.load(std::memory_order_relaxed); }
 void set_sm_budget(int sms) { g_sm_budget.store(sms, std::memory_order_relaxed); }
+std::atomic<int> g_lm_head_pairing{0};
+int lm_head_pairing() { return g_lm_head_pairing.load(std::memory_order_relaxed); }
+void set_lm_head_pairing(int on) { g_lm_head_pairing.store(on != 0 ? 1 : 0, std::memory_order_relaxed); }
 
 rpx_status_t check_arch() {
     int dev = 0, major = 0;

@@ -20,6 +20,8 @@ rpx_status_t encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, cons
 int sm_count();                 // multiprocessors of the current device (cached per device)
 int sm_budget();                // process-wide cap on persistent grids; 0 = none
 void set_sm_budget(int sms);
+int lm_head_pairing();          // process-wide: 1 = the LM head runs its CTA-pair (cta_group::2) kernel
+void set_lm_head_pairing(int on);
 rpx_status_t check_arch();      // RPX_OK on compute capability 10.x
 
 // f32 -> bf16 (round to nearest even) of `rows` rows of `cols` contiguous elements.

@@ -271,6 +271,226 @@ lm_head_partial_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     if (threadIdx.x == 0 && ctl->abort_flag != 0u && p.status != nullptr) atomicCAS(p.status, 0, RPX_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2): a cluster of two CTAs computes a 256-row x 256-column tile.  Each CTA loads its own
+// 128 rows of hidden states and HALF of the W tile (128 of the 256 vocabulary rows), so a stage is 32 KB instead of
+// 48 KB per CTA: a third less L2 -> SM and shared-memory traffic per flop, and six stages in the same shared memory.
+// The even CTA issues the MMAs for both (M = 256); each CTA's four epilogue warps read their own 128 TMEM lanes.
+//   full[s]       lives in the even CTA: its producer arms it with the bytes of BOTH CTAs' loads, and both CTAs'
+//                 TMA loads complete on it
+//   empty[s], tmem_full[a]   live in each CTA; the even CTA's issuer signals both copies with one multicast commit
+//   tmem_empty[a] lives in the even CTA: one arrival per epilogue warp of either CTA (the odd CTA's arrive remotely)
+constexpr int kPairStages = 6;
+constexpr int kPairBBytes = 128 * kBK * 2;
+constexpr int kPairStageBytes = kABytes + kPairBBytes;
+
+struct PairCtl {
+    uint64_t full[kPairStages];
+    uint64_t empty[kPairStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+    uint32_t drain_flag;
+};
+constexpr size_t kPairSmemBytes = 1024 + static_cast<size_t>(kPairStages) * kPairStageBytes + sizeof(PairCtl);
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+lm_head_partial_pair_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
+                            const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    // both CTAs of a pair must use the same offsets: the dynamic window starts at the same shared-memory address in
+    // every CTA of a launch, so rounding it up gives the same result in both
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem_a = smem;
+    uint8_t* smem_b = smem + kPairStages * kABytes;
+    PairCtl* ctl = reinterpret_cast<PairCtl*>(smem + kPairStages * kPairStageBytes);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0 = the CTA that issues the MMAs
+    const int32_t pair = static_cast<int32_t>(blockIdx.x >> 1), n_pairs = static_cast<int32_t>(gridDim.x >> 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&ctl->tmem_full[a], 1);
+            mbar_init(&ctl->tmem_empty[a], 8);  // four epilogue warps in each CTA
+        }
+        mbar_init(&ctl->drain, 1);
+        ctl->abort_flag = 0;
+        ctl->drain_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmap_hidden);
+        tma_prefetch_desc(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(&ctl->tmem_base, kTmemCols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything is sent to them
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one thread in each CTA)
+        if (elect_one()) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int32_t idx = pair; ok && idx < p.total_items; idx += n_pairs) {
+                const Item item = decode_item(p, idx);  // m_tile counts 256-row tiles here
+                for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t) {
+                    for (int32_t kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                        const uint32_t stage = it % kPairStages, phase = (it / kPairStages) & 1u;
+                        if (!mbar_wait(&ctl->empty[stage], phase ^ 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        if (rank == 0) mbar_arrive_expect_tx(&ctl->full[stage], 2 * kPairStageBytes);
+                        const uint32_t full0 = mapa_u32(smem_u32(&ctl->full[stage]), 0);
+                        tma_load_2d_pair(smem_a + stage * kABytes, &tmap_hidden, full0, kb * kBK,
+                                         (item.m_tile * 2 + static_cast<int32_t>(rank)) * kBM);
+                        tma_load_2d_pair(smem_b + stage * kPairBBytes, &tmap_w, full0, kb * kBK,
+                                         t * kBN + static_cast<int32_t>(rank) * (kBN / 2));
+                    }
+                }
+            }
+            if (!ok && rank == 0) {
+                const uint32_t first = it > kPairStages ? it - kPairStages : 0u;
+                for (uint32_t j = first; j < it; ++j)
+                    mbar_wait(&ctl->full[j % kPairStages], (j / kPairStages) & 1u, &ctl->drain_flag, kDrainLimitCycles);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (one thread of the even CTA)
+        if (rank == 0 && elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(2 * kBM, kBN, false, false);
+            const uint64_t a_desc0 = make_smem_desc_sw128(smem_u32(smem_a), 16, 1024);
+            const uint64_t b_desc0 = make_smem_desc_sw128(smem_u32(smem_b), 16, 1024);
+            uint32_t it = 0, tile_count = 0;
+            bool ok = true;
+            for (int32_t idx = pair; ok && idx < p.total_items; idx += n_pairs) {
+                const Item item = decode_item(p, idx);
+                for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
+                    const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(&ctl->tmem_empty[acc], acc_phase ^ 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + acc * kBN;
+                    for (int32_t kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                        const uint32_t stage = it % kPairStages, phase = (it / kPairStages) & 1u;
+                        if (!mbar_wait(&ctl->full[stage], phase, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        umma_pair_ss_k64(d_tmem, a_desc0 + static_cast<uint64_t>(stage * (kABytes >> 4)),
+                                         b_desc0 + static_cast<uint64_t>(stage * (kPairBBytes >> 4)), idesc, kb != 0 ? 1u : 0u);
+                        umma_commit_pair(&ctl->empty[stage], 3);  // the stage is free in both CTAs
+                    }
+                    if (ok) umma_commit_pair(&ctl->tmem_full[acc], 3);
+                }
+            }
+            if (!ok) {
+                umma_commit(&ctl->drain);
+                mbar_wait(&ctl->drain, 0, &ctl->drain_flag, kDrainLimitCycles);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (128 threads in each CTA)
+        const uint32_t quarter = warp & 3;
+        const int32_t row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (quarter * 32u) << 16;
+        uint32_t tile_count = 0;
+        bool ok = true;
+        for (int32_t idx = pair; ok && idx < p.total_items; idx += n_pairs) {
+            const Item item = decode_item(p, idx);
+            const int64_t row = (static_cast<int64_t>(item.m_tile) * 2 + rank) * kBM + row_in_tile;
+            const bool valid = row < p.n_rows;
+            const int32_t target = valid ? __ldg(p.target_ids + row) - p.target_offset : -1;
+            float run_max = -CUDART_INF_F, run_sum = 0.f, target_logit = 0.f, run_wsum = 0.f;
+            for (int32_t t = item.tile_begin; ok && t < item.tile_end; ++t, ++tile_count) {
+                const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+                if (!mbar_wait(&ctl->tmem_full[acc], acc_phase, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const int32_t n0 = t * kBN;
+#pragma unroll 1
+                for (int c = 0; c < kBN / 32; ++c) {
+                    const int32_t col0 = n0 + c * 32;
+                    if (col0 >= p.vocab) break;
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + acc * kBN + c * 32 + lane_addr, r);
+                    tmem_ld_wait();
+                    float x[32];
+                    float cmax = -CUDART_INF_F;
+                    if (col0 + 32 <= p.vocab) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            x[i] = __uint_as_float(r[i]) * kLog2e;
+                            cmax = fmaxf(cmax, x[i]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            x[i] = (col0 + i < p.vocab) ? __uint_as_float(r[i]) * kLog2e : -CUDART_INF_F;
+                            cmax = fmaxf(cmax, x[i]);
+                        }
+                    }
+                    const uint32_t tl = static_cast<uint32_t>(target - col0);
+                    if (tl < 32u) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (tl == static_cast<uint32_t>(i)) target_logit = __uint_as_float(r[i]);
+                    }
+                    const float new_max = fmaxf(run_max, cmax);
+                    const float shrink = fast_exp2(run_max - new_max);
+                    run_sum *= shrink;
+                    run_wsum *= shrink;
+                    float part = 0.f, wpart = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float e = fast_exp2(x[i] - new_max);
+                        part += e;
+                        wpart = fmaf(e, __uint_as_float(r[i]), wpart);
+                    }
+                    run_sum += part;
+                    run_wsum += wpart;
+                    run_max = new_max;
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&ctl->tmem_empty[acc]), 0));
+            }
+            if (ok && valid)
+                p.partials[static_cast<int64_t>(item.chunk) * p.n_rows + row] =
+                    make_float4(run_max, run_sum, target_logit, run_wsum);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA leaves, or frees TMEM, while the other may still signal or read
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+    if (threadIdx.x == 0 && ctl->abort_flag != 0u && p.status != nullptr) atomicCAS(p.status, 0, RPX_ERR_TIMEOUT);
+}
+
 __global__ void lm_head_combine_kernel(const float4* __restrict__ partials, int32_t n_chunks, int64_t n_rows,
                                        const int32_t* __restrict__ target_ids, int32_t vocab,
                                        float* __restrict__ logprobs, float* __restrict__ lse,
@@ -375,11 +595,30 @@ rpx_status_t launch_token_logprobs(const LogprobArgs& a) {
     p.partials = static_cast<float4*>(a.partials);
     p.status = a.device_status;
 
-    if (cudaFuncSetAttribute(lm_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(kSmemBytes)) != cudaSuccess)  // per device, cheap: set every time
-        return RPX_ERR_CUDA;
-    lm_head_partial_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w, p);
-    if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    if (lm_head_pairing() != 0 && sms >= 2) {
+        // CTA pairs: the work list runs over 256-row tiles, the W map hands out half tiles of 128 vocabulary rows
+        CUtensorMap tmap_w_half;
+        const uint64_t dims[2] = {static_cast<uint64_t>(a.hidden_dim), static_cast<uint64_t>(a.vocab)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a.hidden_dim) * 2};
+        const uint32_t box[2] = {kBK, kBN / 2};
+        if (rpx_status_t rc = encode_tmap_bf16(&tmap_w_half, a.w, 2, dims, strides, box)) return rc;
+        p.n_row_tiles = (p.n_row_tiles + 1) / 2;
+        const int64_t total_pairs = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
+        p.total_items = static_cast<int32_t>(total_pairs);
+        const int pairs = static_cast<int>(total_pairs < sms / 2 ? total_pairs : sms / 2);
+        p.group_width = (pairs % 4 == 0 && p.n_row_tiles > kSmallRowTiles / 2) ? 4 : (pairs % 2 == 0 ? 2 : 1);
+        if (cudaFuncSetAttribute(lm_head_partial_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kPairSmemBytes)) != cudaSuccess)
+            return RPX_ERR_CUDA;
+        lm_head_partial_pair_kernel<<<2 * pairs, kThreads, kPairSmemBytes, a.stream>>>(tmap_h, tmap_w_half, p);
+        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    } else {
+        if (cudaFuncSetAttribute(lm_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSmemBytes)) != cudaSuccess)  // per device, cheap: set every time
+            return RPX_ERR_CUDA;
+        lm_head_partial_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w, p);
+        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+    }
     const int cthreads = 256;
     const unsigned cblocks = static_cast<unsigned>((a.n_tokens + cthreads - 1) / cthreads);
     lm_head_combine_kernel<<<cblocks, cthreads, 0, a.stream>>>(p.partials, p.n_chunks, a.n_tokens, a.target_ids,

@@ -236,6 +236,75 @@ __device__ __forceinline__ void umma_ts_k128(uint32_t tmem_d, uint32_t tmem_a, u
         : "memory");
 }
 
+// ------------------------------------------------------------------------------ CTA pairs (cta_group::2)
+// Two CTAs of a cluster of two work on one 256-row MMA tile: each holds its own 128 rows of A, half of the N rows
+// of B and its own 128 TMEM lanes of D; the even CTA issues the MMAs for both.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {  // every thread of both CTAs
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on a barrier given by its shared::cluster address
+// (the even CTA's barrier, for both CTAs of a pair).  No multicast: each CTA fetches its own tile.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint32_t mbar_cluster_addr, int32_t c0,
+                                                 int32_t c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(mbar_cluster_addr), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {  // one warp in EACH CTA
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// One arrival on the barrier at this shared-memory offset in every CTA of `cta_mask`, once the MMAs issued so far
+// by this thread have completed.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                     smem_u32(bar)),
+                 "h"(cta_mask)
+                 : "memory");
+}
+// Four K=16 steps inside one 64-element swizzled K block, M = 256 over the CTA pair: D (+)= A * B.
+__device__ __forceinline__ void umma_pair_ss_k64(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate_first) {
+#define RPX_UMMA2_SS_STEP(off)                                                 \
+    "add.s64 da, %1, " #off ";\n"                                              \
+    "add.s64 db, %2, " #off ";\n"                                              \
+    "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pt;\n"
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 pf, %4, 0;\n"
+        "setp.eq.b32 pt, %4, %4;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pf;\n" RPX_UMMA2_SS_STEP(2) RPX_UMMA2_SS_STEP(4)
+            RPX_UMMA2_SS_STEP(6) "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+#undef RPX_UMMA2_SS_STEP
+}
+
 // 32 lanes x 32 columns of 32-bit: thread t of the warp receives columns c..c+31 of lane (base+t).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(

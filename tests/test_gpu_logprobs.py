@@ -160,3 +160,37 @@ def test_entropy_from_the_same_pass(cuda_device, n_tokens, hidden, vocab, scale)
     got = ent.double().cpu().numpy()
     assert np.isfinite(got).all() and (got > -1e-3).all() and (got < np.log(vocab) + 1e-3).all()
     assert np.abs(got - ref).max() <= TIGHT + 1e-5 * np.abs(ref).max() * (scale > 1)
+
+
+@pytest.mark.parametrize("n_tokens,hidden,vocab", [
+    (300, 200, 1000),     # three row tiles: the second 256-row tile is half empty
+    (1, 8, 3),
+    (129, 72, 257),
+    (640, 1024, 33000),
+    (5000, 512, 20000),   # more work items than CTA pairs
+])
+def test_cta_pair_kernel_matches_the_oracle_and_the_single_cta_kernel(cuda_device, n_tokens, hidden, vocab):
+    """The cta_group::2 variant of the LM head (two CTAs per 256 x 256 tile): same oracle, same bound, and - since each
+    row's products are accumulated in the same order and folded by the same epilogue - the same bits as the
+    single-CTA kernel, entropy included."""
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, hidden, vocab, ("fixed", n_tokens), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=5, attn=False)
+    h, w, ids = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    assert not rpx.get_lm_head_pairing()
+    ent_a = torch.empty(n_tokens, dtype=torch.float32, device=dev)
+    lp_a, lse_a = rpx.token_logprobs(h, w, ids, return_lse=True, entropy=ent_a, device_status=status)
+    try:
+        rpx.set_lm_head_pairing(True)
+        assert rpx.get_lm_head_pairing()
+        ent_b = torch.empty(n_tokens, dtype=torch.float32, device=dev)
+        lp_b, lse_b = rpx.token_logprobs(h, w, ids, return_lse=True, entropy=ent_b, device_status=status)
+        torch.cuda.synchronize()
+    finally:
+        rpx.set_lm_head_pairing(False)
+    assert int(status.item()) == 0
+    ref_lp, ref_lse = oracle.logprob_rows(wl.hidden, wl.w, wl.ids)
+    assert np.abs(lp_b.double().cpu().numpy() - ref_lp).max() <= TIGHT
+    assert np.abs(lse_b.double().cpu().numpy() - ref_lse).max() <= TIGHT
+    assert torch.equal(lp_a, lp_b) and torch.equal(lse_a, lse_b) and torch.equal(ent_a, ent_b)
