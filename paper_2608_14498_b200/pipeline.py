@@ -17,6 +17,28 @@ from . import binding as B
 KERNELS_PER_SCORE = 6  # prefix attn, suffix attn, 2 x (LM-head partial + combine)
 
 
+def backward_through_boundary(q, k, v, out, attn_lse, cu_seqlens, prompt_lens, max_seqlen: int, w_vocab, target_ids,
+                              lm_lse, upstream, softmax_scale: float = 0.0, device_status=None):
+    """Backward of the scoring chain of a training actor whose prefix stays attached (Section 3.2), for the chained
+    case in which the LM head reads the attention output (hidden = out viewed as [tokens, H_q * d]).
+
+    Call order, all arithmetic in the library: (1) the LM head's gradient with respect to its hidden rows from the
+    saved lse; (2) the SUFFIX pass's attention backward - the response rows only - which leaves its additions on the
+    prompt's K/V as well as on the responses' own; (3) the PREFIX pass's attention backward - the prompt rows - added on
+    top.  Whole sequences (prompt followed by response) packed by ``cu_seqlens``; ``prompt_lens`` int32 [B] on the
+    device.  Returns (dq of the response rows, dq of the prompt rows, dk, dv): float32, the two dq tensors are zero
+    outside their own rows."""
+    hidden = out.reshape(out.shape[0], out.shape[1] * out.shape[2])
+    dh = B.token_logprobs_backward(hidden, w_vocab, target_ids, lm_lse, upstream, device_status=device_status)
+    dout = dh.reshape(out.shape)
+    dq_s, dk, dv = B.attn_backward(q, k, v, out, dout, attn_lse, cu_seqlens, max_seqlen, q_begin=prompt_lens,
+                                   softmax_scale=softmax_scale, device_status=device_status)
+    dq_p, dk, dv = B.attn_backward(q, k, v, out, dout, attn_lse, cu_seqlens, max_seqlen, q_end=prompt_lens,
+                                   softmax_scale=softmax_scale, dk=dk, dv=dv, accumulate_dkv=True,
+                                   device_status=device_status)
+    return dq_s, dq_p, dk, dv
+
+
 @dataclass
 class Batch:
     """Tensors of one batch (all on one device, or all pinned host tensors).
