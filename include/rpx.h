@@ -265,7 +265,8 @@ RPX_API size_t rpx_token_logprobs_backward_workspace_bytes(int64_t n_tokens, int
  *       prefix pass's call leaves the same sums as one call over all rows
  *   workspace: rpx_attn_backward_workspace_bytes (D, 4 bytes per token and query head), 256-byte aligned
  * P and dS are rounded to bf16 before they enter the tensor-core products, as P is in the forward pass.
- * cu_seqlens that leave the packed tensors are not followed and set RPX_ERR_DEVICE_DATA in *device_status.
+ * cu_seqlens that leave the packed tensors are not followed and set RPX_ERR_DEVICE_DATA in *device_status; so does a
+ * sequence longer than max_seqlen rounded up to 128 (its rows beyond the bound take no part).
  */
 RPX_API rpx_status_t rpx_attn_backward(const rpx_attn_desc_t* desc, const void* q, const void* k, const void* v,
                                        int64_t q_tok_stride, int64_t k_tok_stride, int64_t v_tok_stride, const void* out,

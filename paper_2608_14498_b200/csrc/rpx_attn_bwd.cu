@@ -240,7 +240,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_x1, const __grid_consta
         uint32_t n_items = 0, n_in = 0;
         for (int32_t rnd = 0, idx = blockIdx.x; ok && idx < p.n_items; idx = item_of_round(++rnd)) {
             const Item it = decode_item<kDq>(p, idx);
-            if (it.bad) ctl->data_error = 1u;  // offsets that leave the packed tensors: reported, not followed
+            // offsets that leave the packed tensors are reported, not followed; so is a sequence longer than the caller's
+            // bound, whose rows beyond it the work list never reaches
+            if (it.bad || it.len > p.n_tiles * kTile) ctl->data_error = 1u;
             if (!it.active) continue;
             const int32_t kv_head = kDq ? it.head / p.group : it.head;
             if (n_items > 0 && !mbar_wait(&ctl->outer_empty, (n_items - 1) & 1u, abort_flag)) {

@@ -181,6 +181,26 @@ def test_sequence_offsets_that_leave_the_tensors_are_reported(cuda_device):
     assert float(dq[200:].abs().max()) == 0.0 and float(dk[200:].abs().max()) == 0.0
 
 
+def test_a_sequence_longer_than_the_callers_bound_is_reported(cuda_device):
+    dev = cuda_device
+    lens, hq, hkv, d = [100, 400], 2, 1, 64
+    q, k, v, dout, cu = _batch(lens, hq, hkv, d, 560)
+    tq, tk, tv, tdo, tcu = (to_device(x, dev) for x in (q, k, v, dout, cu))
+    out, lse = _forward(dev, tq, tk, tv, tcu, 400)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    rpx.attn_backward(tq, tk, tv, out, tdo, lse, tcu, 256, device_status=status)   # 400 > 256
+    torch.cuda.synchronize()
+    assert int(status.item()) == -8
+    status.zero_()
+    rpx.attn_backward(tq, tk, tv, out, tdo, lse, tcu, 300, device_status=status)   # 300 rounds up to 384, still short of 400
+    torch.cuda.synchronize()
+    assert int(status.item()) == -8
+    status.zero_()
+    rpx.attn_backward(tq, tk, tv, out, tdo, lse, tcu, 390, device_status=status)   # 390 rounds up to 512 >= 400
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+
 def test_c2_at_full_size_against_the_oracle_on_one_kv_group(cuda_device):
     """The benchmark's backward workload (C2: 8 whole sequences of 4352 tokens, 28 query / 4 KV heads, head_dim 128)
     through the same call the benchmark times; the oracle differentiates one (sequence, KV head) slice - attention
