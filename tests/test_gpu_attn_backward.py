@@ -181,6 +181,27 @@ def test_sequence_offsets_that_leave_the_tensors_are_reported(cuda_device):
     assert float(dq[200:].abs().max()) == 0.0 and float(dk[200:].abs().max()) == 0.0
 
 
+EDGE = [1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 383, 385]
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_batches_with_random_row_ranges(cuda_device, case):
+    rng = np.random.default_rng(3000 + case)
+    group, hkv = int(rng.integers(1, 9)), int(rng.integers(1, 4))
+    d = 128 if case % 3 else 64
+    batch = int(rng.integers(1, 6))
+    lens = [int(rng.choice(EDGE)) if rng.random() < 0.6 else int(rng.integers(0, 420)) for _ in range(batch)]
+    if sum(lens) == 0:
+        lens[0] = 5
+    q_begin = q_end = None
+    if case % 3 == 1:    # suffix-pass shape: a prompt length per sequence
+        q_begin = [int(rng.integers(0, n + 1)) for n in lens]
+    elif case % 3 == 2:  # arbitrary windows, some empty, some reaching outside
+        q_begin = [int(rng.integers(-3, n + 2)) for n in lens]
+        q_end = [int(rng.integers(-3, n + 5)) for n in lens]
+    _run(cuda_device, lens, group * hkv, hkv, d, 3100 + case, q_begin=q_begin, q_end=q_end)
+
+
 def test_a_sequence_longer_than_the_callers_bound_is_reported(cuda_device):
     dev = cuda_device
     lens, hq, hkv, d = [100, 400], 2, 1, 64
