@@ -2,7 +2,7 @@
 """Benchmark of the prefix+suffix scoring hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3]
-    python bench.py --profile-case lm|lmbwd|prefix|suffix|attnbwd [--reps 3]      (small launches for profiler captures)
+    python bench.py --profile-case lm|lmbwd|lmdw|prefix|suffix|attnbwd [--reps 3]      (small launches for profiler captures)
     python bench.py --attn-alone [--reps 30]                             (attention passes of C2, C3, C4 timed alone)
 
 One step = one pass of the whole path over one synthetic batch: prefix attention (+ paged
@@ -402,11 +402,34 @@ def measure_backward(torch, config, local_rank, reps=3):
     ms = e0.elapsed_time(e1) / reps
     peaks = load_peaks()
     tf = 4.0 * n * cfg.hidden * cfg.vocab / (ms * 1e-3) / 1e12
+    # the same call with the weight gradient as well (a third GEMM over the same block-wise dL/dz)
+    dw = torch.empty((cfg.vocab, cfg.hidden), dtype=torch.float32, device=dev)
+    rpx.token_logprobs_backward(h, w, ids, lse, g, dhidden=dh, dw=dw, workspace=ws, device_status=status)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(gpu_id)
+    time.sleep(0.3)
+    sampler.mark()
+    e0.record()
+    for _ in range(reps):
+        rpx.token_logprobs_backward(h, w, ids, lse, g, dhidden=dh, dw=dw, workspace=ws, device_status=status)
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.mark()
+    clocks_dw = sampler.stop()
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} in the backward pass")
+    ms_dw = e0.elapsed_time(e1) / reps
+    tf_dw = 6.0 * n * cfg.hidden * cfg.vocab / (ms_dw * 1e-3) / 1e12
+    sustained = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     return {"what": "rpx_token_logprobs_backward on the prompt rows (dL/dz from the saved lse, then dlogits x W)",
             "workload": cfg.name, "rows": n, "ms": ms, "tflops": tf,
-            "frac_of_sustained_peak": tf / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+            "frac_of_sustained_peak": tf / sustained,
             "frac_of_burst_peak": tf / float(peaks["bf16_tflops"]), "workspace_bytes": ws.numel(),
-            "gpu_launches": 2 * reps * -(-n // 9472), "clocks": clocks}
+            "gpu_launches": 2 * reps * -(-n // 9472), "clocks": clocks,
+            "with_weight_gradient": {"what": "rpx_token_logprobs_backward_full: dhidden and dW (6 * N * H * V flops)",
+                                     "ms": ms_dw, "tflops": tf_dw, "frac_of_sustained_peak": tf_dw / sustained,
+                                     "frac_of_burst_peak": tf_dw / float(peaks["bf16_tflops"]),
+                                     "gpu_launches": 3 * reps * -(-n // 9472), "clocks": clocks_dw}}
 
 
 def measure_attn_backward(torch, config, local_rank, reps=60):
@@ -529,6 +552,7 @@ def run_profile_case(args):
     after one warm-up launch.
       lm      8192 rows x 32768 vocabulary columns, hidden 3584  (7B-shaped slice of the LM head)
       lmbwd   the same slice through rpx_token_logprobs_backward (two kernels per launch: dL/dz, then dhidden)
+      lmdw    the same with the weight gradient as well (three kernels per launch: dL/dz, dhidden, dW)
       prefix  4 sequences x 4096 prompt tokens, 28 query / 4 KV heads, head_dim 128, with cache write
       suffix  the same 4 prompts cached, 256 response tokens each
       attnbwd rpx_attn_backward over the same 4 sequences whole (4352 tokens each): D, two clears, the dK/dV kernel,
@@ -552,14 +576,15 @@ def run_profile_case(args):
         h, w, ids = dv(wl.hidden), dv(wl.w), dv(wl.ids)
         for _ in range(1 + args.reps):
             rpx.token_logprobs(h, w, ids, device_status=status)
-    elif case == "lmbwd":
+    elif case in ("lmbwd", "lmdw"):
         cfg = wk.Config("profile-lm", "bf16", 1, 28, 4, 128, 3584, 32768, ("fixed", 8192), ("fixed", 0))
         wl = wk.make_workload(cfg, seed=0, attn=False)
         h, w, ids = dv(wl.hidden), dv(wl.w), dv(wl.ids)
         _, lse = rpx.token_logprobs(h, w, ids, return_lse=True, device_status=status)
         g = torch.ones(h.shape[0], dtype=torch.float32, device=dev)
+        dw = torch.empty((w.shape[0], w.shape[1]), dtype=torch.float32, device=dev) if case == "lmdw" else None
         for _ in range(1 + args.reps):
-            rpx.token_logprobs_backward(h, w, ids, lse, g, device_status=status)
+            rpx.token_logprobs_backward(h, w, ids, lse, g, dw=dw, device_status=status)
     elif case == "attnbwd":
         cfg = wk.Config("profile-attn", "bf16", 4, 28, 4, 128, 3584, 1024, ("fixed", 4096), ("fixed", 256))
         wl = wk.make_workload(cfg, seed=0, lm=False)
@@ -743,7 +768,7 @@ def main():
     ap.add_argument("--config", default="C3", choices=sorted(wk.CONFIGS), help="headline workload (C3 = the largest single-GPU config)")
     ap.add_argument("--no-sub-configs", action="store_true", help="skip the C2 / C4 / C5 records of the `configs` key")
     ap.add_argument("--no-backward", action="store_true", help="skip the LM-head backward record (key `backward`)")
-    ap.add_argument("--profile-case", choices=["lm", "lmbwd", "prefix", "suffix", "attnbwd"], help="launch one kernel a few times on a small case and exit")
+    ap.add_argument("--profile-case", choices=["lm", "lmbwd", "lmdw", "prefix", "suffix", "attnbwd"], help="launch one kernel a few times on a small case and exit")
     ap.add_argument("--lm-head-pairing", action="store_true",
                     help="run the LM head's CTA-pair (cta_group::2) kernel instead of the single-CTA one")
     ap.add_argument("--attn-alone", action="store_true", help="time the attention passes of C2, C3 and C4 alone (--reps launches each)")

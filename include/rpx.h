@@ -231,13 +231,27 @@ RPX_API rpx_status_t rpx_token_logprobs_merge(const float* shard_stats, int32_t 
  *   workspace: rpx_token_logprobs_backward_workspace_bytes; it holds dL/dz of one block of at most 9472 rows as
  *   bf16 (9472 x 152064 x 2 bytes = 2.9 GB for the 152064-column vocabulary), never of the whole batch.
  * A target outside [0, vocab) contributes no one-hot term and sets RPX_ERR_DEVICE_DATA in *device_status.
- * The weight gradient is not produced by this call.
+ *
+ * rpx_token_logprobs_backward_full also produces the weight gradient from the same block-wise dL/dz:
+ *     dw[v,:] = sum_n dL/dz[n,v] * hidden[n,:]
+ *   dhidden  as above, or NULL to skip it
+ *   dw       device float32 [vocab][hidden_dim] contiguous, 16-byte aligned, or NULL to skip it (at least one of the
+ *            two must be given); accumulate_dw == 0: written, != 0: the call's gradient is ADDED to what dw holds
+ *            (gradient accumulation over micro-batches)
+ * The contraction runs over the rows, so both operands are read as MN-major tiles straight from the row-major dL/dz
+ * block and hidden tensor.  rpx_token_logprobs_backward is the same call with dw == NULL.
  */
 RPX_API rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
                                                  const int32_t* target_ids, const float* lse, const float* upstream,
                                                  int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype,
                                                  void* dhidden, void* workspace, size_t workspace_bytes,
                                                  int32_t* device_status, void* cuda_stream);
+RPX_API rpx_status_t rpx_token_logprobs_backward_full(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                                      const int32_t* target_ids, const float* lse, const float* upstream,
+                                                      int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
+                                                      rpx_dtype_t dtype, void* dhidden, float* dw, int32_t accumulate_dw,
+                                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                                      void* cuda_stream);
 RPX_API size_t rpx_token_logprobs_backward_workspace_bytes(int64_t n_tokens, int32_t hidden_dim, int32_t vocab,
                                                            rpx_dtype_t dtype);
 

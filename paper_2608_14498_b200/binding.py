@@ -28,6 +28,7 @@ EXPORTS = (
     "rpx_token_logprobs_merge",
     "rpx_token_logprobs_static",
     "rpx_token_logprobs_backward",
+    "rpx_token_logprobs_backward_full",
     "rpx_token_logprobs_backward_workspace_bytes",
     "rpx_set_lm_head_pairing",
     "rpx_get_lm_head_pairing",
@@ -108,6 +109,8 @@ def load_library():
     lib.rpx_token_logprobs_static.argtypes = [vp, i64, vp, vp, i64, i32, i32, vp, vp, vp, vp]
     lib.rpx_token_logprobs_backward.restype = i32
     lib.rpx_token_logprobs_backward.argtypes = [vp, i64, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.rpx_token_logprobs_backward_full.restype = i32
+    lib.rpx_token_logprobs_backward_full.argtypes = [vp, i64, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, i32, vp, sz, vp, vp]
     lib.rpx_token_logprobs_backward_workspace_bytes.restype = sz
     lib.rpx_token_logprobs_backward_workspace_bytes.argtypes = [i64, i32, i32, i32]
     lib.rpx_attn_backward.restype = i32
@@ -396,10 +399,13 @@ def token_logprobs_backward_workspace_bytes(n_tokens, hidden_dim, vocab, dtype_c
 
 @_in_call_context
 def token_logprobs_backward(hidden, w_vocab, target_ids, lse, upstream, dhidden=None, workspace=None, device_status=None,
-                            stream=None):
-    """rpx_token_logprobs_backward: d(sum upstream * logprobs) / d hidden, bf16 [N, H].
+                            stream=None, dw=None, want_dw: bool = False, accumulate_dw: bool = False,
+                            want_dhidden: bool = True):
+    """rpx_token_logprobs_backward(_full): d(sum upstream * logprobs) / d hidden, bf16 [N, H], and - with ``want_dw`` or a
+    ``dw`` buffer - d / d w_vocab, float32 [V, H] (added to ``dw`` when ``accumulate_dw``).
 
-    ``lse`` is the forward call's lse output for the same rows, ``upstream`` float32 [N]."""
+    ``lse`` is the forward call's lse output for the same rows, ``upstream`` float32 [N].  Returns dhidden, or
+    (dhidden, dw) when the weight gradient was asked for (dhidden is None with ``want_dhidden=False``)."""
     torch = _torch()
     lib = load_library()
     if _dtype_code(hidden) != RPX_BF16 or _dtype_code(w_vocab) != RPX_BF16:
@@ -410,15 +416,24 @@ def token_logprobs_backward(hidden, w_vocab, target_ids, lse, upstream, dhidden=
         raise TypeError("lse and upstream are float32")
     n, hdim = hidden.shape
     vocab = w_vocab.shape[0]
-    if dhidden is None:
+    if dhidden is None and want_dhidden:
         dhidden = torch.empty((n, hdim), dtype=torch.bfloat16, device=hidden.device)
+    with_dw = want_dw or dw is not None
+    if with_dw:
+        if dw is None:
+            if accumulate_dw:
+                raise ValueError("accumulate_dw needs the dw buffer to add to")
+            dw = torch.empty((vocab, hdim), dtype=torch.float32, device=hidden.device)
+        if dw.dtype != torch.float32 or not dw.is_contiguous() or tuple(dw.shape) != (vocab, hdim):
+            raise ValueError("dw is a contiguous float32 [V, H] tensor")
     ws = _workspace(int(lib.rpx_token_logprobs_backward_workspace_bytes(n, hdim, vocab, RPX_BF16)), hidden.device, workspace)
-    rc = lib.rpx_token_logprobs_backward(_ptr(hidden), hidden.stride(0) if n > 1 else hdim, _ptr(w_vocab), _ptr(target_ids),
-                                         _ptr(lse), _ptr(upstream), n, hdim, vocab, RPX_BF16, _ptr(dhidden), _ptr(ws),
-                                         ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
+    rc = lib.rpx_token_logprobs_backward_full(_ptr(hidden), hidden.stride(0) if n > 1 else hdim, _ptr(w_vocab),
+                                              _ptr(target_ids), _ptr(lse), _ptr(upstream), n, hdim, vocab, RPX_BF16,
+                                              _ptr(dhidden), _ptr(dw), 1 if accumulate_dw else 0, _ptr(ws),
+                                              ws.numel() * ws.element_size(), _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
-        raise RpxError(rc, "rpx_token_logprobs_backward")
-    return dhidden
+        raise RpxError(rc, "rpx_token_logprobs_backward_full")
+    return (dhidden, dw) if with_dw else dhidden
 
 
 @_in_call_context

@@ -259,22 +259,22 @@ size_t rpx_token_logprobs_backward_workspace_bytes(int64_t n_tokens, int32_t hid
     return align_up(logprob_backward_workspace(n_tokens, vocab), kWsAlign);
 }
 
-rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
-                                         const int32_t* target_ids, const float* lse, const float* upstream,
-                                         int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype,
-                                         void* dhidden, void* workspace, size_t workspace_bytes, int32_t* device_status,
-                                         void* cuda_stream) {
+rpx_status_t rpx_token_logprobs_backward_full(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                              const int32_t* target_ids, const float* lse, const float* upstream,
+                                              int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype,
+                                              void* dhidden, float* dw, int32_t accumulate_dw, void* workspace,
+                                              size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
     if (dtype != RPX_BF16 && dtype != RPX_F32) return RPX_ERR_DTYPE;
     if (dtype != RPX_BF16) return RPX_ERR_DTYPE;  // the backward pass takes bf16 tensors only
     if (n_tokens < 0 || n_tokens >= INT32_MAX || hidden_dim <= 0 || vocab <= 0) return RPX_ERR_SHAPE;
     if (hidden_dim % 8 != 0) return RPX_ERR_SHAPE;
     if (n_tokens == 0) return RPX_OK;
     if (hidden == nullptr || w_vocab == nullptr || target_ids == nullptr || lse == nullptr || upstream == nullptr ||
-        dhidden == nullptr)
+        (dhidden == nullptr && dw == nullptr))
         return RPX_ERR_NULL;
     if (hidden_row_stride < hidden_dim) return RPX_ERR_SHAPE;
     if (hidden_row_stride % 8 != 0) return RPX_ERR_ALIGN;
-    if (!aligned16(hidden) || !aligned16(w_vocab) || !aligned16(dhidden)) return RPX_ERR_ALIGN;
+    if (!aligned16(hidden) || !aligned16(w_vocab) || !aligned16(dhidden) || !aligned16(dw)) return RPX_ERR_ALIGN;
     const size_t need = rpx_token_logprobs_backward_workspace_bytes(n_tokens, hidden_dim, vocab, dtype);
     if (workspace == nullptr || workspace_bytes < need) return RPX_ERR_WORKSPACE;
     if (!aligned_ws(workspace)) return RPX_ERR_ALIGN;
@@ -290,10 +290,24 @@ rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_
     a.hidden_dim = hidden_dim;
     a.vocab = vocab;
     a.dhidden = dhidden;
+    a.dw = dw;
+    a.accumulate_dw = accumulate_dw != 0;
     a.dlogits = workspace;
     a.device_status = device_status;
     a.stream = static_cast<cudaStream_t>(cuda_stream);
     return launch_token_logprobs_backward(a);
+}
+
+rpx_status_t rpx_token_logprobs_backward(const void* hidden, int64_t hidden_row_stride, const void* w_vocab,
+                                         const int32_t* target_ids, const float* lse, const float* upstream,
+                                         int64_t n_tokens, int32_t hidden_dim, int32_t vocab, rpx_dtype_t dtype,
+                                         void* dhidden, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                         void* cuda_stream) {
+    if (dtype == RPX_BF16 && n_tokens > 0 && hidden_dim > 0 && vocab > 0 && hidden_dim % 8 == 0 && dhidden == nullptr)
+        return RPX_ERR_NULL;
+    return rpx_token_logprobs_backward_full(hidden, hidden_row_stride, w_vocab, target_ids, lse, upstream, n_tokens,
+                                            hidden_dim, vocab, dtype, dhidden, nullptr, 0, workspace, workspace_bytes,
+                                            device_status, cuda_stream);
 }
 
 size_t rpx_attn_backward_workspace_bytes(const rpx_attn_desc_t* desc, int64_t total_tokens) {

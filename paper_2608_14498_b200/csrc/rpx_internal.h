@@ -88,7 +88,9 @@ struct LogprobBwdArgs {
     const float* upstream;     // [n], dL / d logprob
     int64_t n_tokens;
     int32_t hidden_dim, vocab;
-    void* dhidden;             // bf16 [n][hidden_dim]
+    void* dhidden;             // bf16 [n][hidden_dim], nullable
+    float* dw = nullptr;       // fp32 [vocab][hidden_dim], nullable
+    bool accumulate_dw = false;  // add dW to what the buffer holds
     void* dlogits;             // workspace: bf16 [logprob_backward_block_rows(n)][vocab rounded up to 64]
     int32_t* device_status;
     cudaStream_t stream;

@@ -14,6 +14,10 @@
 //                    weight, exactly as V is taken in the attention kernel; never transposed, never copied.
 // CTAs resident together cover (block row tiles) x (4 output-column tiles) and walk the vocabulary in step, so
 // every dlogits and W tile is pulled from HBM once per wave and shared through L2.
+//   dW kernel        (optional) dlogits^T x hidden: the contraction runs over the block's rows, so BOTH operands are
+//                    MN-major - dlogits [rows][vocab] with the vocabulary as M, hidden [rows][H] with H as N - again
+//                    straight from their row-major tensors; 128 vocabulary rows x 256 columns of W's gradient per
+//                    tile, written (first block) or added (later blocks) as fp32.
 //
 // Warp roles as in the forward kernel (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
@@ -64,6 +68,8 @@ struct Params {
     int64_t dlogits_stride;
     __nv_bfloat16* dhidden;     // [n_rows][dhidden_stride]
     int64_t dhidden_stride;
+    float* dw;                  // dW kernel: [vocab][hidden_dim]
+    int32_t dw_add;             // add to what dw holds (every block after the first, or the caller's request)
     int32_t* status;
 };
 
@@ -110,9 +116,35 @@ __device__ __forceinline__ void umma_ss_k64_bmn(uint32_t tmem_d, uint64_t adesc,
         : "memory");
 }
 
-// kDhidden = false: the dlogits kernel (A = hidden, B = W K-major over hidden_dim, epilogue = dL/dz to the workspace)
-// kDhidden = true : the dhidden kernel (A = dlogits, B = W MN-major over the vocabulary, epilogue = bf16 tile out)
-template <bool kDhidden>
+// Four K=16 steps of D (+)= A[smem, MN-major] * B[smem, MN-major]: both advance 16 rows of 128 bytes (128 units).
+__device__ __forceinline__ void umma_ss_k64_amn_bmn(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                    uint32_t accumulate_first) {
+    asm volatile(
+        "{\n"
+        ".reg .pred pf, pt;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 pf, %4, 0;\n"
+        "setp.eq.b32 pt, %4, %4;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n"
+        "add.s64 da, %1, 128;\n"
+        "add.s64 db, %2, 128;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n"
+        "add.s64 da, %1, 256;\n"
+        "add.s64 db, %2, 256;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n"
+        "add.s64 da, %1, 384;\n"
+        "add.s64 db, %2, 384;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n"
+        "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first)
+        : "memory");
+}
+
+// kMode 0: the dlogits kernel (A = hidden, B = W K-major over hidden_dim, epilogue = dL/dz to the workspace)
+// kMode 1: the dhidden kernel (A = dlogits, B = W MN-major over the vocabulary, epilogue = bf16 tile out)
+// kMode 2: the dW kernel      (A = dlogits MN-major with the vocabulary as M, B = hidden MN-major, contraction over
+//                              the block's rows, epilogue = fp32 tile of W's gradient, written or added)
+template <int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -124,7 +156,8 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int32_t tiles_per_item = kDhidden ? 1 : kTilesPerChunk;
+    constexpr bool kDhidden = kMode == 1, kDw = kMode == 2;
+    const int32_t tiles_per_item = kMode == 0 ? kTilesPerChunk : 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -168,9 +201,17 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                             break;
                         }
                         mbar_arrive_expect_tx(&ctl->full[stage], kABytes + kBBytes);
-                        tma_load_2d(smem_a + stage * kABytes, &tmap_a, &ctl->full[stage], kb * kBK, item.m_tile * kBM);
-                        if (kDhidden) {
-                            // W [V][H] as {H, V}: four boxes of 64 output columns x 64 vocabulary rows
+                        if (kDw) {
+                            // dlogits [rows][vocab] as {vocab, rows}: two boxes of 64 vocabulary columns x 64 rows
+                            for (int i = 0; i < kBM / 64; ++i)
+                                tma_load_2d(smem_a + stage * kABytes + i * (kBK * 128), &tmap_a, &ctl->full[stage],
+                                            item.m_tile * kBM + i * 64, kb * kBK);
+                        } else {
+                            tma_load_2d(smem_a + stage * kABytes, &tmap_a, &ctl->full[stage], kb * kBK, item.m_tile * kBM);
+                        }
+                        if (kDhidden || kDw) {
+                            // W [V][H] as {H, V} (dW: hidden [rows][H] as {H, rows}): four boxes of 64 output columns x
+                            // 64 rows of the contraction
                             for (int i = 0; i < kBN / 64; ++i)
                                 tma_load_2d(smem_b + stage * kBBytes + i * (kBK * 128), &tmap_b, &ctl->full[stage],
                                             t * kBN + i * 64, kb * kBK);
@@ -191,10 +232,10 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (one thread)
         if (elect_one()) {
-            constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, false, kDhidden);
-            const uint64_t a_desc0 = make_smem_desc_sw128(smem_u32(smem_a), 16, 1024);
-            // MN-major B: 64-column blocks lie kBK rows of 128 bytes apart
-            const uint64_t b_desc0 = make_smem_desc_sw128(smem_u32(smem_b), kDhidden ? kBK * 128 : 16, 1024);
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, kDw, kDhidden || kDw);
+            // MN-major operands: 64-element blocks of M (or N) lie kBK rows of 128 bytes apart
+            const uint64_t a_desc0 = make_smem_desc_sw128(smem_u32(smem_a), kDw ? kBK * 128 : 16, 1024);
+            const uint64_t b_desc0 = make_smem_desc_sw128(smem_u32(smem_b), (kDhidden || kDw) ? kBK * 128 : 16, 1024);
             uint32_t it = 0, tile_count = 0;
             bool ok = true;
             for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
@@ -217,7 +258,8 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                         tc_fence_after_sync();
                         const uint64_t ad = a_desc0 + static_cast<uint64_t>(stage * (kABytes >> 4));
                         const uint64_t bd = b_desc0 + static_cast<uint64_t>(stage * (kBBytes >> 4));
-                        if (kDhidden) umma_ss_k64_bmn(d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u);
+                        if (kDw) umma_ss_k64_amn_bmn(d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u);
+                        else if (kDhidden) umma_ss_k64_bmn(d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u);
                         else umma_ss_k64(d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u);
                         umma_commit(&ctl->empty[stage]);
                     }
@@ -240,10 +282,10 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         for (int32_t idx = blockIdx.x; ok && idx < p.total_items; idx += gridDim.x) {
             const Item item = decode_item(p, idx);
             const int64_t row = static_cast<int64_t>(item.m_tile) * kBM + row_in_tile;
-            const bool valid = row < p.n_rows;
+            const bool valid = kDw ? row < p.vocab : row < p.n_rows;  // dW: the tile's rows are vocabulary rows
             int32_t target = -1;
             float lse2 = 0.f, g = 0.f;
-            if (!kDhidden && valid) {
+            if (kMode == 0 && valid) {
                 target = __ldg(p.target_ids + row);
                 if (target < 0 || target >= p.vocab) {
                     ctl->data_error = 1;  // no one-hot term for such a row (its log-prob is NaN in the forward pass)
@@ -261,7 +303,7 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 }
                 tc_fence_after_sync();
                 const int32_t n0 = t * kBN;
-                const int32_t n_cols = kDhidden ? p.hidden_dim : p.vocab;
+                const int32_t n_cols = kMode == 0 ? p.vocab : p.hidden_dim;
                 __nv_bfloat16* dst_row = kDhidden ? p.dhidden + row * p.dhidden_stride : p.dlogits + row * p.dlogits_stride;
 #pragma unroll 1
                 for (int c = 0; c < kBN / 32; ++c) {
@@ -270,6 +312,29 @@ lm_head_bwd_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     uint32_t r[32];
                     tmem_ld32(tmem_base + acc * kBN + c * 32 + lane_addr, r);
                     tmem_ld_wait();
+                    if (kDw) {
+                        // fp32 tile of W's gradient; hidden_dim is a multiple of 8, so whole groups of 4 columns
+                        if (valid) {
+                            float* dst = p.dw + row * p.hidden_dim + col0;
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                if (col0 + i < n_cols) {
+                                    float4 v = make_float4(__uint_as_float(r[i]), __uint_as_float(r[i + 1]),
+                                                           __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                                    float4* q4 = reinterpret_cast<float4*>(dst + i);
+                                    if (p.dw_add != 0) {
+                                        const float4 old = *q4;
+                                        v.x += old.x;
+                                        v.y += old.y;
+                                        v.z += old.z;
+                                        v.w += old.w;
+                                    }
+                                    *q4 = v;
+                                }
+                            }
+                        }
+                        continue;
+                    }
                     uint32_t w[16];
                     if (kDhidden) {
 #pragma unroll
@@ -340,9 +405,11 @@ rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a) {
     int sms = sm_count();
     if (sms <= 0) return RPX_ERR_CUDA;
     if (const int budget = sm_budget(); budget > 0 && budget < sms) sms = budget;  // leave the rest to a co-runner
-    if (cudaFuncSetAttribute(lm_head_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(lm_head_bwd_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(kSmemBytes)) != cudaSuccess ||
-        cudaFuncSetAttribute(lm_head_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(lm_head_bwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kSmemBytes)) != cudaSuccess ||
+        cudaFuncSetAttribute(lm_head_bwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(kSmemBytes)) != cudaSuccess)
         return RPX_ERR_CUDA;
     const int64_t block_rows = logprob_backward_block_rows(a.n_tokens);
@@ -363,7 +430,7 @@ rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a) {
     }
     for (int64_t r0 = 0; r0 < a.n_tokens; r0 += block_rows) {
         const int64_t rows = a.n_tokens - r0 < block_rows ? a.n_tokens - r0 : block_rows;
-        CUtensorMap tmap_h, tmap_dl;
+        CUtensorMap tmap_h, tmap_dl, tmap_h_mn, tmap_dl_mn;
         {
             const uint64_t dims[2] = {static_cast<uint64_t>(a.hidden_dim), static_cast<uint64_t>(rows)};
             const uint64_t strides[1] = {static_cast<uint64_t>(a.hidden_row_stride) * 2};
@@ -376,7 +443,20 @@ rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a) {
             const uint32_t box[2] = {kBK, kBM};
             if (rpx_status_t rc = encode_tmap_bf16(&tmap_dl, dlogits, 2, dims, strides, box)) return rc;
         }
+        if (a.dw != nullptr) {
+            // the dW kernel's views: boxes of 64 contiguous elements (vocabulary columns of dlogits, columns of hidden)
+            // x 64 rows of the block; rows beyond the block read as zero
+            const uint32_t box[2] = {64, kBK};
+            const uint64_t hdims[2] = {static_cast<uint64_t>(a.hidden_dim), static_cast<uint64_t>(rows)};
+            const uint64_t hstrides[1] = {static_cast<uint64_t>(a.hidden_row_stride) * 2};
+            if (rpx_status_t rc = encode_tmap_bf16(&tmap_h_mn, hidden + r0 * a.hidden_row_stride, 2, hdims, hstrides, box)) return rc;
+            const uint64_t ddims[2] = {static_cast<uint64_t>(a.vocab), static_cast<uint64_t>(rows)};
+            const uint64_t dstrides[1] = {static_cast<uint64_t>(dl_stride) * 2};
+            if (rpx_status_t rc = encode_tmap_bf16(&tmap_dl_mn, dlogits, 2, ddims, dstrides, box)) return rc;
+        }
         Params p;
+        p.dw = a.dw;
+        p.dw_add = (a.accumulate_dw || r0 > 0) ? 1 : 0;
         p.n_rows = rows;
         p.vocab = a.vocab;
         p.hidden_dim = a.hidden_dim;
@@ -398,18 +478,35 @@ rpx_status_t launch_token_logprobs_backward(const LogprobBwdArgs& a) {
         p.total_items = static_cast<int32_t>(total);
         int grid = static_cast<int>(total < sms ? total : sms);
         p.group_width = grid % 4 == 0 ? 4 : (grid % 2 == 0 ? 2 : 1);
-        lm_head_bwd_kernel<false><<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w_k, p);
+        lm_head_bwd_kernel<0><<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_h, tmap_w_k, p);
         if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
         // ---- dhidden of the block
-        p.k_blocks = (a.vocab + kBK - 1) / kBK;
-        p.n_col_tiles = (a.hidden_dim + kBN - 1) / kBN;
-        p.n_chunks = p.n_col_tiles;
-        total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
-        p.total_items = static_cast<int32_t>(total);
-        grid = static_cast<int>(total < sms ? total : sms);
-        p.group_width = p.n_col_tiles % 4 == 0 ? 4 : (p.n_col_tiles % 2 == 0 ? 2 : 1);
-        lm_head_bwd_kernel<true><<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_dl, tmap_w_mn, p);
-        if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+        if (a.dhidden != nullptr) {
+            p.k_blocks = (a.vocab + kBK - 1) / kBK;
+            p.n_col_tiles = (a.hidden_dim + kBN - 1) / kBN;
+            p.n_chunks = p.n_col_tiles;
+            total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
+            p.total_items = static_cast<int32_t>(total);
+            grid = static_cast<int>(total < sms ? total : sms);
+            p.group_width = p.n_col_tiles % 4 == 0 ? 4 : (p.n_col_tiles % 2 == 0 ? 2 : 1);
+            lm_head_bwd_kernel<1><<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_dl, tmap_w_mn, p);
+            if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+        }
+        // ---- this block's share of dW: the work list runs over (128 vocabulary rows) x (256 columns of hidden_dim),
+        // all column tiles of a vocabulary tile side by side, so a dlogits slice is pulled from HBM once
+        if (a.dw != nullptr) {
+            p.k_blocks = static_cast<int32_t>((rows + kBK - 1) / kBK);
+            p.n_row_tiles = (a.vocab + kBM - 1) / kBM;
+            p.n_col_tiles = (a.hidden_dim + kBN - 1) / kBN;
+            p.n_chunks = p.n_col_tiles;
+            total = static_cast<int64_t>(p.n_row_tiles) * p.n_chunks;
+            if (total > INT32_MAX) return RPX_ERR_SHAPE;
+            p.total_items = static_cast<int32_t>(total);
+            grid = static_cast<int>(total < sms ? total : sms);
+            p.group_width = p.n_col_tiles <= 20 ? p.n_col_tiles : 16;
+            lm_head_bwd_kernel<2><<<grid, kThreads, kSmemBytes, a.stream>>>(tmap_dl_mn, tmap_h_mn, p);
+            if (cudaGetLastError() != cudaSuccess) return RPX_ERR_CUDA;
+        }
     }
     return RPX_OK;
 }

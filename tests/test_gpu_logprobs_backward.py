@@ -94,3 +94,54 @@ def test_backward_rejects_bad_arguments_before_any_launch(cuda_device):
     assert call(h=100) == -2 and call(stride=128) == -2
     assert call(ws=None) == -5 and call(ws_bytes=64) == -5 and call(ws=0x10010) == -4
     assert call(n=0, hidden=None) == 0
+
+
+def _dw_close(got, ref):
+    got = got.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    # dL/dz passes through bf16 (2^-9 relative per term) before the products are summed over the rows in fp32
+    bound = 0.01 * np.abs(ref).max() + np.abs(ref) * 2.0 ** -7 + 1e-7
+    err = np.abs(got - ref)
+    assert (err <= bound).all(), f"dW: max err {err.max():.3e} of max |ref| {np.abs(ref).max():.3e}"
+
+
+@pytest.mark.parametrize("n_tokens,hidden,vocab", [(288, 256, 4096), (130, 72, 1000), (1, 64, 257), (700, 512, 9000),
+                                                   (300, 200, 255), (257, 128, 64)])
+def test_weight_gradient_matches_the_oracle(cuda_device, n_tokens, hidden, vocab):
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, hidden, vocab, ("fixed", n_tokens), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=81, attn=False)
+    h, w, tid = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    g = np.random.default_rng(82).standard_normal(n_tokens).astype(np.float32)
+    tg = torch.from_numpy(g).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    _, lse = rpx.token_logprobs(h, w, tid, return_lse=True, device_status=status)
+    dh_only = rpx.token_logprobs_backward(h, w, tid, lse, tg, device_status=status)
+    dh, dw = rpx.token_logprobs_backward(h, w, tid, lse, tg, want_dw=True, device_status=status)
+    none, dw_only = rpx.token_logprobs_backward(h, w, tid, lse, tg, want_dw=True, want_dhidden=False, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert none is None and torch.equal(dh, dh_only) and torch.equal(dw, dw_only)
+    _, ref_dw = oracle.logprob_backward(wl.hidden, wl.w, wl.ids, g.astype(np.float64), want_dw=True)
+    _dw_close(dw, ref_dw)
+    # gradient accumulation: a second call adds its gradient to the buffer
+    dw2 = dw.clone()
+    rpx.token_logprobs_backward(h, w, tid, lse, tg, dw=dw2, accumulate_dw=True, want_dhidden=False, device_status=status)
+    torch.cuda.synchronize()
+    _dw_close(dw2, 2.0 * ref_dw)
+
+
+def test_weight_gradient_over_more_rows_than_one_block(cuda_device):
+    dev = cuda_device
+    n_tokens, hidden, vocab = 9472 + 300, 64, 320   # the second block of rows adds to the first one's dW
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, hidden, vocab, ("fixed", n_tokens), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=83, attn=False)
+    h, w, tid = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    g = np.random.default_rng(84).standard_normal(n_tokens).astype(np.float32)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    _, lse = rpx.token_logprobs(h, w, tid, return_lse=True, device_status=status)
+    _, dw = rpx.token_logprobs_backward(h, w, tid, lse, torch.from_numpy(g).to(dev), want_dw=True, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    _, ref_dw = oracle.logprob_backward(wl.hidden, wl.w, wl.ids, g.astype(np.float64), want_dw=True)
+    _dw_close(dw, ref_dw)
