@@ -15,6 +15,8 @@
 //               O_t += P_t V  (P_t = bf16 probabilities written back into the first 64 columns
 //               of S_t's TMEM region and consumed as the TMEM A operand; V straight from its
 //               [keys][d] tile as an MN-major B operand)
+//   warps 10-11: fill the producer's and the issuer's warp group: after setup that group hands most of its registers
+//               to the two softmax warp groups (setmaxnreg), whose step keeps 128 scores and their exponentials live
 // The two query tiles alternate on the tensor core in the order PV_0(j) QK_0(j+1) PV_1(j)
 // QK_1(j+1): while the softmax warps of one tile work on S_t, the tensor core runs the other
 // tile's two MMAs; issuing PV_t(j) before QK_t(j+1) also orders the read of P_t before the
@@ -38,7 +40,15 @@ constexpr int kItemRing = 4;  // work-item ids the producer may hand out ahead o
 constexpr int kChunks = kTileK / 32;  // 32-column TMEM loads per row and step
 constexpr int kWarpsPerTile = 4;
 constexpr int kProducerWarp = 2 * kWarpsPerTile, kMmaWarp = kProducerWarp + 1;
-constexpr int kThreads = 32 * (kMmaWarp + 1);
+// Three warp groups of four: the eight softmax warps, then the producer, the issuer and two warps that only take part
+// in the register hand-over (setmaxnreg works on whole warp groups).
+constexpr int kThreads = 32 * 12;
+// Registers per thread after the hand-over (256 softmax threads, 128 others; the SM has 65536).  The prefix pass's
+// branch-free softmax step wants as many as it can get (208 + 80); in passes over cached tiles the producer's paged
+// loads set the pace and it must not be squeezed (184 + 128): measured, the other way round loses 3 - 7 % each.
+template <bool kFastSteps> struct Regs {
+    static constexpr int kSoftmax = kFastSteps ? 208 : 184, kOther = kFastSteps ? 80 : 128;
+};
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -191,7 +201,9 @@ __device__ __forceinline__ Item decode_item(const Params& p, int4 rec) {
     return it;
 }
 
-template <int D>
+// kFastSteps: also instantiate the branch-free form of the softmax step (see there); the launcher picks it for the
+// prefix pass.
+template <int D, bool kFastSteps>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
             const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_kc,
@@ -252,9 +264,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
     // TMEM columns: S_t at 128 t (P_t aliases its first 64), O_t at 256 + 128 t
+    // The kernel starts with 168 registers per thread (65536 / 384); the producer / issuer warp group gives most of
+    // its share to the two softmax warp groups, whose step keeps 128 scores and their exponentials in flight.
+    // (each role states its new count at the top of its own branch, which is where the compiler looks for it)
 
     if (warp == kProducerWarp) {
         // =========================================================== producer warp
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Regs<kFastSteps>::kOther));
         bool ok = true;
         if (lane == 0) {
             tma_prefetch_desc(&tmap_q);
@@ -446,6 +462,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
         }
     } else if (warp == kMmaWarp) {
         // =========================================================== tcgen05 issuer (one thread)
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Regs<kFastSteps>::kOther));
         if (elect_one()) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(kTileQ, kTileK, false, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(kTileQ, D, false, true);
@@ -558,8 +575,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
             }
         }
         __syncwarp();
+    } else if (warp > kMmaWarp) {
+        // warps 10 and 11: nothing to do between the register hand-over and the teardown
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(Regs<kFastSteps>::kOther));
     } else {
         // =========================================================== softmax warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(Regs<kFastSteps>::kSoftmax));
         const int t = warp / kWarpsPerTile;
         uint32_t n_seen = 0;  // work items read from the item ring
         uint32_t cnt = 0;     // key steps this tile has been through (barrier parity)
@@ -624,7 +645,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     const int32_t jt = j - n_prefix_tiles;
                     n_vis = min(kTileK, max(0, q_local - jt * kTileK + 1));
                 }
-                if (n_vis < kTileK) {
+                // The step's arithmetic exists twice: the general form masks the scores a row may not see and skips
+                // whole chunks nobody in the warp sees; the fast form, for tiles every row of the warp sees completely
+                // (the self tiles left of the diagonal), has neither test, so the unrolled step is one basic block the
+                // compiler can schedule across.  Only the prefix pass's instance of the kernel has it: passes over cached
+                // tiles run at the pace of the producer's page-sized loads, and there the second copy of the step
+                // measured 2 - 7 % slower.
+                float alpha = 1.f;
+                bool rescale = false;
+                auto body = [&](auto fast_tag) {
+                constexpr bool kFast = decltype(fast_tag)::value;
+                if (!kFast && n_vis < kTileK) {
 #pragma unroll
                     for (int c = 0; c < kChunks; ++c)
 #pragma unroll
@@ -633,7 +664,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 }
                 // keys no row of this warp may see (the upper right of a diagonal tile, the tail of the last
                 // prefix tile) need no exponentials: their 32-column chunks get P = 0 directly
-                const int32_t n_vis_warp = __reduce_max_sync(0xffffffffu, n_vis);
+                const int32_t n_vis_warp = kFast ? kTileK : __reduce_max_sync(0xffffffffu, n_vis);
                 // eight independent chains of three-input maxima (the maximum runs on the half-rate ALU pipe,
                 // so halving its instruction count is worth more than it looks)
                 float mx[8];
@@ -650,8 +681,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 // an integer maximum can be folded exactly into the rounding constant of the polynomial exp2 below.
                 const bool grow = cmax > run_max + kRescaleThreshold;
                 const float new_max = grow ? ceilf(cmax) : run_max;
-                const float alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
-                const bool rescale = j > 0 && __any_sync(0xffffffffu, grow);
+                alpha = grow ? fast_exp2(run_max - new_max) : 1.f;
+                rescale = j > 0 && __any_sync(0xffffffffu, grow);
                 run_sum *= alpha;
                 run_max = new_max;
                 // ---- P = 2^(x - max) as packed bf16 pairs over the first 64 columns of S_t
@@ -667,7 +698,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     for (int c = 0; c < kChunks; ++c) {
                         uint32_t packed[16];
                         uint32_t lo[4];
-                        if (c * 32 >= n_vis_warp) {
+                        if (!kFast && c * 32 >= n_vis_warp) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) packed[i] = 0u;
                             tmem_st16(my_s + c * 16, packed);
@@ -720,6 +751,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                     f2_unpack(f2_add(f2_add(part2[0], part2[1]), f2_add(part2[2], part2[3])), a0, a1);
                     run_sum += a0 + a1;
                 }
+                };
+                if (kFastSteps && !kSplit && __all_sync(0xffffffffu, n_vis == kTileK)) body(std::true_type{});
+                else body(std::false_type{});
                 // S_t(j) was committed behind PV_t(j-1), so O_t is quiescent until this warp's arrival
                 // below.  Done here,
                 // after the scores are dead, so the 32 staging registers do not force spills.
@@ -1010,10 +1044,12 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     const int sms = sms_all;  // SM count, or the caller's SM budget: the rest is left to a co-runner
     const int64_t grid = n_items < sms ? n_items : sms;  // persistent: one CTA per SM
     if (cudaMemsetAsync(a.item_counter, 0, sizeof(uint32_t), a.stream) != cudaSuccess) return RPX_ERR_CUDA;
-    if (cudaFuncSetAttribute(attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(L::kSmemBytes)) != cudaSuccess)
+    // the prefix pass (no cached tiles) runs the instance with the branch-free softmax step
+    auto* kernel = a.prefix_lens == nullptr ? attn_kernel<D, true> : attn_kernel<D, false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(L::kSmemBytes)) !=
+        cudaSuccess)
         return RPX_ERR_CUDA;
-    attn_kernel<D><<<static_cast<unsigned>(grid), kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tkc, tvc, p);
+    kernel<<<static_cast<unsigned>(grid), kThreads, L::kSmemBytes, a.stream>>>(tq, tk, tv, tkc, tvc, p);
     return cudaGetLastError() == cudaSuccess ? RPX_OK : RPX_ERR_CUDA;
 }
 
