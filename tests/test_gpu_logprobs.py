@@ -194,3 +194,32 @@ def test_cta_pair_kernel_matches_the_oracle_and_the_single_cta_kernel(cuda_devic
     assert np.abs(lp_b.double().cpu().numpy() - ref_lp).max() <= TIGHT
     assert np.abs(lse_b.double().cpu().numpy() - ref_lse).max() <= TIGHT
     assert torch.equal(lp_a, lp_b) and torch.equal(lse_a, lse_b) and torch.equal(ent_a, ent_b)
+
+
+def test_cta_pair_kernel_under_an_sm_budget_and_through_the_other_entry_points(cuda_device):
+    """The pair kernel runs whole clusters only: an odd SM budget leaves one SM unused, a budget of one falls back to
+    the single-CTA kernel; the shard and static entry points take the same switch."""
+    dev = cuda_device
+    cfg = wk.Config("t", "bf16", 1, 1, 1, 64, 256, 3000, ("fixed", 700), ("fixed", 0))
+    wl = wk.make_workload(cfg, seed=6, attn=False)
+    h, w, ids = to_device(wl.hidden, dev), to_device(wl.w, dev), to_device(wl.ids, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ref = rpx.token_logprobs(h, w, ids, device_status=status)
+    try:
+        rpx.set_lm_head_pairing(True)
+        for budget in (0, 7, 2, 1):
+            rpx.set_sm_budget(budget)
+            got = rpx.token_logprobs(h, w, ids, device_status=status)
+            torch.cuda.synchronize()
+            assert torch.equal(got, ref), budget
+        rpx.set_sm_budget(0)
+        lp = torch.empty(700, dtype=torch.float32, device=dev)
+        rpx.token_logprobs_static(h, w, ids, lp, device_status=status)
+        stats = rpx.token_logprobs_shard(h, w[:1500], ids, 0, device_status=status)
+        torch.cuda.synchronize()
+        assert float((lp - ref).abs().max()) <= 2e-5   # the static entry point always uses 16-tile chunks: another merge order
+        assert stats.shape == (700, 4) and bool(torch.isfinite(stats).all())
+    finally:
+        rpx.set_sm_budget(0)
+        rpx.set_lm_head_pairing(False)
+    assert int(status.item()) == 0
