@@ -181,6 +181,27 @@ def test_sequence_offsets_that_leave_the_tensors_are_reported(cuda_device):
     assert float(dq[200:].abs().max()) == 0.0 and float(dk[200:].abs().max()) == 0.0
 
 
+def test_peaked_rows_and_a_long_sequence(cuda_device):
+    dev = cuda_device
+    # scores a few tens apart: most rows put their weight on one or two keys, P is 1 or ~0 and dS nearly cancels
+    lens, hq, hkv, d = [300, 200], 4, 2, 64
+    q, k, v, dout, cu = _batch(lens, hq, hkv, d, 570)
+    q = wk.f32_to_bf16_bits(wk.bf16_bits_to_f32(q) * 4.0).reshape(q.shape)   # exact in bf16
+    k = wk.f32_to_bf16_bits(wk.bf16_bits_to_f32(k) * 2.0).reshape(k.shape)
+    tq, tk, tv, tdo, tcu = (to_device(x, dev) for x in (q, k, v, dout, cu))
+    out, lse = _forward(dev, tq, tk, tv, tcu, 300)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    dq, dk, dv = rpx.attn_backward(tq, tk, tv, out, tdo, lse, tcu, 300, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rq, rk, rv = oracle.attn_backward(q, k, v, cu, _masked_dout(dout, cu, None, None))
+    _close(dq, rq, "dq")
+    _close(dk, rk, "dk")
+    _close(dv, rv, "dv")
+    # one long sequence: 40 key tiles, every inner-loop length from 1 to 40
+    _run(dev, [5000], 2, 1, 64, 571)
+
+
 EDGE = [1, 2, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 383, 385]
 
 
