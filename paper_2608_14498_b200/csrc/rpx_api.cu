@@ -90,7 +90,6 @@ rpx_status_t run_attention(const rpx_attn_desc_t* desc, const void* q, const voi
         a.split_ws = static_cast<uint8_t*>(workspace) + kWsAlign;
     a.append_cache = is_suffix && append_cache;
     a.out = out;
-    a.out_f32 = desc->dtype == RPX_F32;
     a.lse = lse;
     a.device_status = device_status;
     a.stream = stream;

@@ -118,8 +118,7 @@ struct Params {
     int64_t total_tokens;
     float scale_log2;
     float inv_scale_log2;
-    void* out;
-    int32_t out_f32;
+    void* out;                    // bf16 [tokens][H_q][D] (fp32 tensors take the CUDA-core kernel)
     float* lse;
     int32_t* status;
 };
@@ -796,22 +795,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ 
                 const bool wide = (reinterpret_cast<uintptr_t>(p.out) & 31u) == 0u;
                 auto store_chunk = [&](const uint32_t (&r)[32], int c) {
                     if (!row_valid) return;
-                    if (p.out_f32) {
-                        float* dst = static_cast<float*>(p.out) + out_row + c * 32;
-                        uint32_t w[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(__uint_as_float(r[i]) * inv);
-                        if (wide) {
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                st_global_v8(dst + 8 * i, w[8 * i], w[8 * i + 1], w[8 * i + 2], w[8 * i + 3], w[8 * i + 4],
-                                             w[8 * i + 5], w[8 * i + 6], w[8 * i + 7]);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-                        }
-                    } else {
+                    {
                         __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.out) + out_row + c * 32;
                         uint32_t w[16];
 #pragma unroll
@@ -998,7 +982,6 @@ rpx_status_t launch_attention_d(const AttnArgs& a) {
     p.scale_log2 = scale * kLog2e;
     p.inv_scale_log2 = 1.0f / p.scale_log2;
     p.out = a.out;
-    p.out_f32 = a.out_f32 ? 1 : 0;
     p.lse = a.lse;
     p.status = a.device_status;
     const int64_t n_base = static_cast<int64_t>(p.n_pairs) * a.batch * p.item_heads;

@@ -42,8 +42,7 @@ struct AttnArgs {
     bool append_cache = false;         // chunked prefill: read the earlier chunks AND append this one
     uint32_t* item_counter = nullptr;  // 4 bytes of workspace: the kernel's work-item counter (zeroed by the launcher)
     void* split_ws = nullptr;          // suffix pass only: room for split-KV partials (attn_split_workspace bytes), or NULL
-    void* out;
-    bool out_f32;
+    void* out;                         // bf16 (launch_attention) or float32 (launch_attention_f32)
     float* lse;
     int32_t* device_status;
     cudaStream_t stream;
